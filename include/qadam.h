@@ -1,0 +1,190 @@
+/*
+ * qadam.h - C interface of the quantized-Adam-with-error-feedback step library
+ * for NVIDIA B200 (sm_100a).
+ *
+ * One context is one parameter-server problem of the paper "Quantized Adam with
+ * Error Feedback": a parameter vector x in R^d (Eq. 1), N workers, a gradient
+ * quantizer Q_g and a weight quantizer Q_x (Section 5.1), Adam parameters
+ * beta, theta, epsilon and a step size alpha_t (Algorithms 1-3).  The N workers
+ * are a batch dimension on one GPU; what a worker would send to the server, and
+ * what the server would broadcast, are packed device buffers.
+ *
+ * Conventions
+ *  - Every pointer in qadam_buffers, and `g`, is a DEVICE pointer owned by the
+ *    caller, 16-byte aligned, valid until qadam_destroy.  The library allocates
+ *    and frees no device memory; its scratch space is `workspace`.
+ *  - Host pointers are marked "host".
+ *  - Calls enqueue work on the context's stream and return without waiting,
+ *    unless stated otherwise.
+ *  - Return value: QADAM_OK, or a negative qadam_error.  On an error nothing
+ *    has been enqueued by that call.  Conditions found on the device (a
+ *    non-finite input, a wait that gave up) set bits of the status word.
+ *  - A context is not thread-safe; distinct contexts are independent.
+ *
+ * Layout ("padded layout")
+ *  The parameter vector is a list of segments (tensors).  Segment s starts at
+ *  element seg_off[s], the running sum of the previous segments' lengths each
+ *  rounded up to a multiple of 128 elements; D is the padded total.  Pad
+ *  elements must be 0 in g, x, m, v, e when the context is created and stay 0.
+ *  Q_g uses one max-abs scale per (worker, segment); num_segments = 1 is the
+ *  paper's literal whole-vector infinity norm.
+ *
+ * Packed streams
+ *  A code is an unsigned integer of b bits; element j of a stream occupies bits
+ *  [j*b, (j+1)*b) of the stream read as a little-endian bit string (bit p is bit
+ *  p mod 8 of byte p / 8).  Gradient code = level index + L, where the level
+ *  index runs over -L..L and L is the number of positive levels of G; weight
+ *  code = level index + 2^kx.  Pads carry level index 0.
+ *  b_g = ceil(log2(2L+1)) (3 levels: 2 bits, 5 levels: 3 bits), b_x = kx + 2:
+ *  the fixed widths behind the "Comm" and "Size" columns of Tables 1-2.
+ *  With kg = -1 (Q_g = identity) the "codes" of a worker are the D binary32
+ *  values it would send and its scales are 1.
+ */
+#ifndef QADAM_H_
+#define QADAM_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct qadam_ctx qadam_ctx;
+
+/* Where Adam's moments m, v live and what Q_g is applied to.
+ *  QADAM_PLACE_WORKER: Algorithms 2-3 as printed.  Each worker keeps its own
+ *    m, v, forms alpha_t m/sqrt(v+eps) + e, quantizes THAT, and the server only
+ *    averages and subtracts.
+ *  QADAM_PLACE_SERVER: the plain distributed Adam the end of Section 3 compares
+ *    with.  Each worker quantizes g + e; the server averages the decoded
+ *    gradients and runs the moment and parameter updates of Algorithm 1. */
+enum { QADAM_PLACE_SERVER = 0, QADAM_PLACE_WORKER = 1 };
+
+/* Reading of the level set G of Section 5.1 for kg >= 2 (identical for kg = 0, 1):
+ *  POW2:    {0, 2^-kg, 2^-kg+1, ..., 1}  (as printed: geometric; L = kg + 1)
+ *  UNIFORM: {0, 1/2^kg, 2/2^kg, ..., 1}  (the spacing printed for X; L = 2^kg) */
+enum { QADAM_GRID_POW2 = 0, QADAM_GRID_UNIFORM = 1 };
+
+enum qadam_error {
+  QADAM_OK = 0,
+  QADAM_ERR_NULL = -1,        /* a required pointer is NULL                         */
+  QADAM_ERR_SIZE = -2,        /* d, n, num_segments or a segment length is invalid  */
+  QADAM_ERR_LEVEL = -3,       /* kg, kx or grid_g outside the supported range       */
+  QADAM_ERR_ALIGN = -4,       /* a device pointer is not 16-byte aligned            */
+  QADAM_ERR_WORKSPACE = -5,   /* workspace_bytes is smaller than qadam_query_sizes says */
+  QADAM_ERR_STEP = -6,        /* step out of order (see the step functions)         */
+  QADAM_ERR_WORKER = -7,      /* worker range outside 0..n                          */
+  QADAM_ERR_HYPER = -8,       /* beta/theta outside [0,1), eps <= 0 or a bad step size */
+  QADAM_ERR_CUDA = -9,        /* a CUDA call failed; see qadam_last_cuda_error      */
+  QADAM_ERR_PLACEMENT = -10   /* placement is not one of the two values             */
+};
+
+/* Bits of the device status word. */
+enum {
+  QADAM_ST_NONFINITE = 1u,    /* a max-abs scale was Inf or NaN: outputs of that step are unspecified */
+  QADAM_ST_TIMEOUT = 2u       /* a bounded wait inside a kernel ran out; outputs of that step are unspecified */
+};
+
+typedef struct {
+  int64_t d;                  /* logical number of parameters (Eq. 1: x in R^d)                 */
+  int32_t n;                  /* N, the number of workers (Algorithms 2-3); 1 gives Algorithm 1 */
+  int32_t num_segments;       /* S >= 1                                                          */
+  const int64_t* seg_len;     /* host, [S], each >= 1, sum = d; may be NULL when S = 1           */
+  int32_t kg;                 /* level parameter of G (Section 5.1), 0 = {-1,0,1}; -1: identity.
+                                 Supported: POW2 0..14, UNIFORM 0..6                            */
+  int32_t kx;                 /* level parameter of X (Section 5.1), 0..14; -1: no weight
+                                 quantization (nothing is broadcast in packed form)             */
+  int32_t grid_g;             /* QADAM_GRID_*                                                    */
+  int32_t placement;          /* QADAM_PLACE_*                                                   */
+  float beta1;                /* beta  of the m update, in [0, 1)                                */
+  float beta2;                /* theta of the v update, in [0, 1)                                */
+  float eps;                  /* epsilon, > 0, added to v INSIDE the square root                 */
+  float lr;                   /* default alpha, used when a step is given a negative lr_t        */
+  void* stream;               /* cudaStream_t all work is enqueued on (NULL: the default stream) */
+} qadam_config;
+
+typedef struct {
+  float* x;                   /* [D] master copy x_t, updated in place                            */
+  float* m;                   /* first moment:  [D] (PLACE_SERVER) or [n][D] (PLACE_WORKER)       */
+  float* v;                   /* second moment: same shape as m                                   */
+  float* e;                   /* [n][D] error-feedback buffers e^(i), updated in place            */
+  float* scales;              /* [n][S] out: max-abs scale of each (worker, segment)              */
+  void* gcodes;               /* [n][gcode_bytes] out: what each worker sends                     */
+  void* wcodes;               /* [wcode_bytes] out: packed Q_x(x); may be NULL when kx = -1       */
+  float* wresid;              /* [D] out, optional (NULL to skip): x - Q_x(x)                     */
+  void* workspace;            /* scratch, workspace_bytes of qadam_query_sizes, 256-byte aligned;
+                                 the library keeps tables here between calls: do not touch it   */
+  size_t workspace_bytes;
+  uint32_t* status;           /* one word; qadam_create clears it                                 */
+} qadam_buffers;
+
+/* Sizes for a configuration.  Any output pointer may be NULL.
+ *  D: padded length; seg_off: host [S] padded segment offsets;
+ *  gcode_bytes: bytes ONE worker sends per step (D*b_g/8, or 4*D when kg = -1);
+ *  wcode_bytes: bytes of the packed broadcast (D*b_x/8, 0 when kx = -1).
+ * Per step the workers send n*(gcode_bytes + 4*S) bytes against 4*d*n unquantized. */
+int qadam_query_sizes(const qadam_config* cfg, int64_t* D, int64_t* seg_off,
+                      size_t* gcode_bytes, size_t* wcode_bytes, size_t* workspace_bytes);
+
+/* Code widths: b_g for (kg, grid_g) (32 when kg = -1), b_x for kx (0 when kx = -1);
+ * negative qadam_error when unsupported. */
+int qadam_grad_code_bits(int32_t kg, int32_t grid_g);
+int qadam_weight_code_bits(int32_t kx);
+
+/* Creates a context.  The caller has put x_1 into x and zeros into m, v, e
+ * (Algorithm 1 / 3: m_0 = v_0 = 0, e_1 = 0).  Writes the library's tables into
+ * the workspace (synchronously) and, when kx >= 0, enqueues the first broadcast
+ * Q_x(x_1) into wcodes (and wresid), the first line of Algorithm 2's loop. */
+int qadam_create(const qadam_config* cfg, const qadam_buffers* bufs, qadam_ctx** out);
+
+/* Worker side of step `step` (1-based) for workers [worker_begin, worker_begin +
+ * worker_count): Algorithm 3, lines from "v = ..." to the error update.
+ *   g: [worker_count][D] stochastic gradients of those workers (padded layout).
+ *   PLACE_WORKER: v, m updates; u = lr_t*m/sqrt(v+eps) + e.   PLACE_SERVER: u = g + e.
+ *   scale = max|u| per segment; codes = nearest level of u/scale in G (ties toward
+ *   zero; all-zero segment: level 0), packed; e <- u - scale*level (Algorithm 1's
+ *   last line).
+ * Steps must be taken in order: `step` must be one more than the last completed
+ * server step, and each worker compresses once per step (not checked: compressing
+ * a worker twice applies the error feedback twice).
+ * lr_t < 0 selects cfg.lr. */
+int qadam_worker_compress(qadam_ctx* ctx, int64_t step, const float* g,
+                          int32_t worker_begin, int32_t worker_count, float lr_t);
+
+/* Server side of step `step`: Algorithm 2's gather-average-update, then the next
+ * broadcast.  Decodes the n streams, delta^ = (sum in worker order 0..n-1)/n,
+ *   PLACE_WORKER: x <- x - delta^              (the printed '+' is read as '-')
+ *   PLACE_SERVER: v, m updates with delta^ as the gradient; x <- x - lr_t*m/sqrt(v+eps)
+ * then, when kx >= 0, wcodes <- packed Q_x(x) (nearest point of the grid of step
+ * 2^-(kx+1) on [-1/2, 1/2], clipped, ties toward zero) and wresid <- x - Q_x(x).
+ * Requires that all n workers were compressed for `step`. */
+int qadam_server_step(qadam_ctx* ctx, int64_t step, float lr_t);
+
+/* One whole step from HOST memory, for callers whose gradients live on the host:
+ * copies g_host ([n][D], host, ideally pinned) into g_stage (device, [n][D],
+ * caller-owned), runs qadam_worker_compress for all workers and
+ * qadam_server_step, then copies the result back to out_host (host): the packed
+ * broadcast (wcode_bytes) when kx >= 0, else x (4*D bytes).  Waits for the
+ * stream before returning.  out_host may be NULL to skip the read-back. */
+int qadam_step_host(qadam_ctx* ctx, int64_t step, const float* g_host, float* g_stage,
+                    void* out_host, float lr_t);
+
+/* Waits for the context's stream, then copies the status word to *host_status. */
+int qadam_poll_status(qadam_ctx* ctx, uint32_t* host_status);
+
+/* Number of kernels this context has launched since it was created. */
+int64_t qadam_launch_count(const qadam_ctx* ctx);
+
+/* Releases the host-side context.  Device buffers stay the caller's. */
+int qadam_destroy(qadam_ctx* ctx);
+
+const char* qadam_strerror(int err);
+
+/* The cudaError_t of the last failed CUDA call made through this library (0 if none). */
+int qadam_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif  /* QADAM_H_ */

@@ -333,8 +333,8 @@ int32_t qo_worker_step(const qo_problem* p, const float* g, float* m, float* v,
     }
     if (p->kg < 0) {
       scales[s] = 1.0f;
-      std::memset(codes + 4 * off, 0, (size_t)(4 * plen));
-      std::memcpy(codes + 4 * off, u.data(), (size_t)(4 * len));
+      u.resize((size_t)plen, 0.0f);                       // pads are sent as zeros
+      std::memcpy(codes + 4 * off, u.data(), sizeof(float) * u.size());
       for (int64_t j = 0; j < len; ++j) e[off + j] = u[j] - u[j];
       continue;
     }

@@ -1,0 +1,423 @@
+// Host side of the C interface declared in include/qadam.h: argument checks,
+// the tile table, launch configuration and the step bookkeeping.  Every step of
+// the method itself runs in the kernels of qadam_kernels.cuh.
+#include "qadam.h"
+
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "qadam_kernels.cuh"
+
+using namespace qadam;
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+inline bool cuda_ok(cudaError_t e) {
+  if (e != cudaSuccess) {
+    g_last_cuda_error = (int)e;
+    return false;
+  }
+  return true;
+}
+
+inline int64_t round_up64(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+int bits_for(int num_codes) {
+  int b = 0;
+  while ((1 << b) < num_codes) ++b;
+  return b;
+}
+
+// Positive levels L of G for (kg, grid), or a negative error.
+int grad_levels(int kg, int grid) {
+  if (grid != QADAM_GRID_POW2 && grid != QADAM_GRID_UNIFORM) return QADAM_ERR_LEVEL;
+  if (kg < 0) return QADAM_ERR_LEVEL;
+  if (kg <= 1) return kg + 1;                          // both grids: {0,1}, {0,1/2,1}
+  if (grid == QADAM_GRID_POW2) return kg <= 14 ? kg + 1 : QADAM_ERR_LEVEL;
+  return kg <= 6 ? (1 << kg) : QADAM_ERR_LEVEL;
+}
+
+struct Geometry {
+  std::vector<int64_t> seg_len, seg_off;
+  int64_t D = 0;
+  std::vector<Tile> tiles;
+  int gbits = 0, xbits = 0, L = 0;
+  GMode gmode = G_TERNARY;
+  size_t gcode_bytes = 0, wcode_bytes = 0, workspace_bytes = 0;
+};
+
+int validate_config(const qadam_config* c) {
+  if (!c) return QADAM_ERR_NULL;
+  if (c->d < 1 || c->n < 1 || c->n > 4096 || c->num_segments < 1) return QADAM_ERR_SIZE;
+  if (c->num_segments > 1 && !c->seg_len) return QADAM_ERR_NULL;
+  if (c->placement != QADAM_PLACE_SERVER && c->placement != QADAM_PLACE_WORKER)
+    return QADAM_ERR_PLACEMENT;
+  if (c->kg < -1 || c->kx < -1 || c->kx > 14) return QADAM_ERR_LEVEL;
+  if (c->kg >= 0 && grad_levels(c->kg, c->grid_g) < 0) return QADAM_ERR_LEVEL;
+  if (c->kg < 0 && c->grid_g != QADAM_GRID_POW2 && c->grid_g != QADAM_GRID_UNIFORM)
+    return QADAM_ERR_LEVEL;
+  if (!(c->beta1 >= 0.0f && c->beta1 < 1.0f) || !(c->beta2 >= 0.0f && c->beta2 < 1.0f) ||
+      !(c->eps > 0.0f) || !std::isfinite(c->eps) || !std::isfinite(c->lr))
+    return QADAM_ERR_HYPER;
+  return QADAM_OK;
+}
+
+int build_geometry(const qadam_config* c, Geometry* g) {
+  int rc = validate_config(c);
+  if (rc != QADAM_OK) return rc;
+  const int S = c->num_segments;
+  g->seg_len.resize(S);
+  g->seg_off.resize(S);
+  int64_t sum = 0, off = 0;
+  for (int s = 0; s < S; ++s) {
+    const int64_t len = (S == 1 && !c->seg_len) ? c->d : c->seg_len[s];
+    if (len < 1) return QADAM_ERR_SIZE;
+    g->seg_len[s] = len;
+    g->seg_off[s] = off;
+    off += round_up64(len, kAlign);
+    sum += len;
+  }
+  if (sum != c->d) return QADAM_ERR_SIZE;
+  g->D = off;
+  if (g->D / kAlign > (int64_t)1 << 30) return QADAM_ERR_SIZE;
+  g->tiles.clear();
+  for (int s = 0; s < S; ++s) {
+    const int64_t plen = round_up64(g->seg_len[s], kAlign);
+    for (int64_t o = 0; o < plen; o += kTileElems) {
+      Tile t;
+      t.off = g->seg_off[s] + o;
+      t.count = (int)std::min<int64_t>(kTileElems, plen - o);
+      t.seg = s;
+      g->tiles.push_back(t);
+    }
+  }
+  if (c->kg < 0) {
+    g->gmode = G_IDENTITY; g->L = 0; g->gbits = 32;
+  } else {
+    g->L = grad_levels(c->kg, c->grid_g);
+    g->gbits = bits_for(2 * g->L + 1);
+    g->gmode = c->kg == 0 ? G_TERNARY : c->kg == 1 ? G_FIVE
+             : c->grid_g == QADAM_GRID_POW2 ? G_POW2 : G_UNIFORM;
+  }
+  g->xbits = c->kx < 0 ? 0 : c->kx + 2;
+  g->gcode_bytes = (size_t)(g->D * g->gbits / 8);
+  g->wcode_bytes = (size_t)(g->D * g->xbits / 8);
+  g->workspace_bytes = (size_t)round_up64((int64_t)g->tiles.size() * sizeof(Tile), 256) + 256;
+  return QADAM_OK;
+}
+
+}  // namespace
+
+struct qadam_ctx {
+  qadam_config cfg;
+  qadam_buffers buf;
+  Geometry geo;
+  Hyper h;
+  cudaStream_t stream;
+  Tile* d_tiles;
+  int sm_count;
+  int64_t last_server_step;     // steps completed by the server
+  int64_t workers_done;         // workers compressed for step last_server_step + 1
+  int64_t launches;
+  int grid_absmax, grid_quant, grid_ident, grid_server, grid_bcast;
+  size_t server_smem;
+};
+
+namespace {
+
+template <typename K>
+int resident_grid(K kernel, size_t smem, int sm_count) {
+  int per_sm = 0;
+  if (!cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, kThreads, smem)))
+    return -1;
+  return std::max(1, per_sm) * sm_count;
+}
+
+using WorkerKernel = void (*)(const WorkerParams);
+using ServerKernel = void (*)(const ServerParams);
+
+WorkerKernel pick_absmax(const qadam_ctx* c) {
+  return c->cfg.placement == QADAM_PLACE_WORKER ? worker_absmax_kernel<true>
+                                                : worker_absmax_kernel<false>;
+}
+
+WorkerKernel pick_identity(const qadam_ctx* c) {
+  return c->cfg.placement == QADAM_PLACE_WORKER ? worker_identity_kernel<true>
+                                                : worker_identity_kernel<false>;
+}
+
+WorkerKernel pick_quantize(const qadam_ctx* c) {
+  const bool w = c->cfg.placement == QADAM_PLACE_WORKER;
+  switch (c->geo.gmode) {
+    case G_TERNARY: return w ? worker_quantize_kernel<true, G_TERNARY> : worker_quantize_kernel<false, G_TERNARY>;
+    case G_FIVE:    return w ? worker_quantize_kernel<true, G_FIVE>    : worker_quantize_kernel<false, G_FIVE>;
+    case G_POW2:    return w ? worker_quantize_kernel<true, G_POW2>    : worker_quantize_kernel<false, G_POW2>;
+    default:        return w ? worker_quantize_kernel<true, G_UNIFORM> : worker_quantize_kernel<false, G_UNIFORM>;
+  }
+}
+
+ServerKernel pick_server(const qadam_ctx* c) {
+  const bool s = c->cfg.placement == QADAM_PLACE_SERVER;
+  switch (c->geo.gmode) {
+    case G_TERNARY:  return s ? server_step_kernel<true, G_TERNARY>  : server_step_kernel<false, G_TERNARY>;
+    case G_FIVE:     return s ? server_step_kernel<true, G_FIVE>     : server_step_kernel<false, G_FIVE>;
+    case G_POW2:     return s ? server_step_kernel<true, G_POW2>     : server_step_kernel<false, G_POW2>;
+    case G_UNIFORM:  return s ? server_step_kernel<true, G_UNIFORM>  : server_step_kernel<false, G_UNIFORM>;
+    default:         return s ? server_step_kernel<true, G_IDENTITY> : server_step_kernel<false, G_IDENTITY>;
+  }
+}
+
+ServerParams make_server_params(const qadam_ctx* c, float alpha) {
+  ServerParams p;
+  p.x = c->buf.x; p.m = c->buf.m; p.v = c->buf.v;
+  p.scales = c->buf.scales;
+  p.gcodes = static_cast<const unsigned char*>(c->buf.gcodes);
+  p.wcodes = static_cast<unsigned char*>(c->buf.wcodes);
+  p.wresid = c->buf.wresid;
+  p.tiles = c->d_tiles;
+  p.D = c->geo.D;
+  p.gcode_bytes = (long long)c->geo.gcode_bytes;
+  p.tiles_per_worker = (int)c->geo.tiles.size();
+  p.S = c->cfg.num_segments;
+  p.n = c->cfg.n;
+  p.k = c->cfg.kg; p.L = c->geo.L; p.gbits = c->geo.gbits;
+  p.kx = c->cfg.kx; p.xbits = c->geo.xbits;
+  p.alpha = alpha;
+  p.nf = (float)c->cfg.n;
+  p.h = c->h;
+  return p;
+}
+
+}  // namespace
+
+extern "C" {
+
+int qadam_grad_code_bits(int32_t kg, int32_t grid_g) {
+  if (kg == -1) return 32;
+  const int L = grad_levels(kg, grid_g);
+  return L < 0 ? L : bits_for(2 * L + 1);
+}
+
+int qadam_weight_code_bits(int32_t kx) {
+  if (kx == -1) return 0;
+  if (kx < 0 || kx > 14) return QADAM_ERR_LEVEL;
+  return kx + 2;
+}
+
+int qadam_query_sizes(const qadam_config* cfg, int64_t* D, int64_t* seg_off,
+                      size_t* gcode_bytes, size_t* wcode_bytes, size_t* workspace_bytes) {
+  Geometry g;
+  const int rc = build_geometry(cfg, &g);
+  if (rc != QADAM_OK) return rc;
+  if (D) *D = g.D;
+  if (seg_off) std::memcpy(seg_off, g.seg_off.data(), g.seg_off.size() * sizeof(int64_t));
+  if (gcode_bytes) *gcode_bytes = g.gcode_bytes;
+  if (wcode_bytes) *wcode_bytes = g.wcode_bytes;
+  if (workspace_bytes) *workspace_bytes = g.workspace_bytes;
+  return QADAM_OK;
+}
+
+int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** out) {
+  if (!cfg || !b || !out) return QADAM_ERR_NULL;
+  *out = nullptr;
+  qadam_ctx* c = new (std::nothrow) qadam_ctx();
+  if (!c) return QADAM_ERR_CUDA;
+  int rc = build_geometry(cfg, &c->geo);
+  if (rc != QADAM_OK) { delete c; return rc; }
+  const bool quant_x = cfg->kx >= 0;
+  if (!b->x || !b->m || !b->v || !b->e || !b->scales || !b->gcodes || !b->workspace ||
+      !b->status || (quant_x && !b->wcodes)) {
+    delete c; return QADAM_ERR_NULL;
+  }
+  const void* ptrs[] = {b->x, b->m, b->v, b->e, b->scales, b->gcodes, b->wcodes, b->wresid, b->status};
+  for (const void* p : ptrs) {
+    if (p && !aligned(p, p == b->status || p == b->scales ? 4 : 16)) { delete c; return QADAM_ERR_ALIGN; }
+  }
+  if (!aligned(b->workspace, 256)) { delete c; return QADAM_ERR_ALIGN; }
+  if (b->workspace_bytes < c->geo.workspace_bytes) { delete c; return QADAM_ERR_WORKSPACE; }
+
+  c->cfg = *cfg;
+  c->cfg.seg_len = nullptr;            // the caller's array is not kept; geo has a copy
+  c->buf = *b;
+  c->stream = static_cast<cudaStream_t>(cfg->stream);
+  c->h.beta = cfg->beta1; c->h.theta = cfg->beta2; c->h.eps = cfg->eps;
+  c->h.one_minus_beta = 1.0f - cfg->beta1;
+  c->h.one_minus_theta = 1.0f - cfg->beta2;
+  c->last_server_step = 0;
+  c->workers_done = 0;
+  c->launches = 0;
+  c->d_tiles = static_cast<Tile*>(b->workspace);
+
+  int dev = 0;
+  if (!cuda_ok(cudaGetDevice(&dev)) ||
+      !cuda_ok(cudaDeviceGetAttribute(&c->sm_count, cudaDevAttrMultiProcessorCount, dev))) {
+    delete c; return QADAM_ERR_CUDA;
+  }
+  c->server_smem = sizeof(float) * (size_t)cfg->n;
+  if (c->geo.gmode != G_TERNARY && c->geo.gmode != G_IDENTITY)
+    c->server_smem += sizeof(float) * (size_t)cfg->n * ((size_t)1 << c->geo.gbits);
+  if (c->server_smem > 200 * 1024) { delete c; return QADAM_ERR_SIZE; }
+  ServerKernel sk = pick_server(c);
+  if (c->server_smem > 48 * 1024 &&
+      !cuda_ok(cudaFuncSetAttribute(sk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->server_smem))) {
+    delete c; return QADAM_ERR_CUDA;
+  }
+  c->grid_absmax = resident_grid(pick_absmax(c), 0, c->sm_count);
+  c->grid_quant = resident_grid(pick_quantize(c), 0, c->sm_count);
+  c->grid_ident = resident_grid(pick_identity(c), 0, c->sm_count);
+  c->grid_server = resident_grid(sk, c->server_smem, c->sm_count);
+  c->grid_bcast = resident_grid(weight_broadcast_kernel, 0, c->sm_count);
+  if (c->grid_absmax < 0 || c->grid_quant < 0 || c->grid_ident < 0 || c->grid_server < 0 ||
+      c->grid_bcast < 0) {
+    delete c; return QADAM_ERR_CUDA;
+  }
+
+  // tables and status: synchronous, so the host vector may go away
+  if (!cuda_ok(cudaMemcpyAsync(c->d_tiles, c->geo.tiles.data(), c->geo.tiles.size() * sizeof(Tile),
+                               cudaMemcpyHostToDevice, c->stream)) ||
+      !cuda_ok(cudaMemsetAsync(b->status, 0, sizeof(uint32_t), c->stream)) ||
+      !cuda_ok(cudaStreamSynchronize(c->stream))) {
+    delete c; return QADAM_ERR_CUDA;
+  }
+  if (quant_x) {
+    const ServerParams p = make_server_params(c, 0.0f);
+    const int grid = (int)std::min<int64_t>(c->grid_bcast, (int64_t)c->geo.tiles.size());
+    weight_broadcast_kernel<<<grid, kThreads, 0, c->stream>>>(p);
+    if (!cuda_ok(cudaGetLastError())) { delete c; return QADAM_ERR_CUDA; }
+    c->launches++;
+  }
+  *out = c;
+  return QADAM_OK;
+}
+
+int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
+                          int32_t worker_begin, int32_t worker_count, float lr_t) {
+  if (!c || !g) return QADAM_ERR_NULL;
+  if (!aligned(g, 16)) return QADAM_ERR_ALIGN;
+  if (step != c->last_server_step + 1) return QADAM_ERR_STEP;
+  if (worker_begin < 0 || worker_count < 1 || (int64_t)worker_begin + worker_count > c->cfg.n)
+    return QADAM_ERR_WORKER;
+  const float alpha = lr_t < 0.0f ? c->cfg.lr : lr_t;
+  if (!std::isfinite(alpha)) return QADAM_ERR_HYPER;
+
+  WorkerParams p;
+  p.g = g;
+  p.m = c->buf.m; p.v = c->buf.v; p.e = c->buf.e;
+  p.scale_bits = reinterpret_cast<unsigned*>(c->buf.scales);
+  p.gcodes = static_cast<unsigned char*>(c->buf.gcodes);
+  p.tiles = c->d_tiles;
+  p.status = c->buf.status;
+  p.D = c->geo.D;
+  p.gcode_bytes = (long long)c->geo.gcode_bytes;
+  p.tiles_per_worker = (int)c->geo.tiles.size();
+  p.total_tiles = (long long)worker_count * p.tiles_per_worker;
+  p.S = c->cfg.num_segments;
+  p.worker_begin = worker_begin;
+  p.k = c->cfg.kg; p.L = c->geo.L; p.bits = c->geo.gbits;
+  p.alpha = alpha;
+  p.h = c->h;
+
+  if (c->geo.gmode == G_IDENTITY) {
+    const int grid = (int)std::min<int64_t>(c->grid_ident, p.total_tiles);
+    pick_identity(c)<<<grid, kThreads, 0, c->stream>>>(p);
+    if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
+    c->launches += 1;
+  } else {
+    if (!cuda_ok(cudaMemsetAsync(p.scale_bits + (size_t)worker_begin * p.S, 0,
+                                 sizeof(unsigned) * (size_t)worker_count * p.S, c->stream)))
+      return QADAM_ERR_CUDA;
+    int grid = (int)std::min<int64_t>(c->grid_absmax, p.total_tiles);
+    pick_absmax(c)<<<grid, kThreads, 0, c->stream>>>(p);
+    if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
+    grid = (int)std::min<int64_t>(c->grid_quant, p.total_tiles);
+    pick_quantize(c)<<<grid, kThreads, 0, c->stream>>>(p);
+    if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
+    c->launches += 2;
+  }
+  c->workers_done += worker_count;
+  return QADAM_OK;
+}
+
+int qadam_server_step(qadam_ctx* c, int64_t step, float lr_t) {
+  if (!c) return QADAM_ERR_NULL;
+  if (step != c->last_server_step + 1 || c->workers_done < c->cfg.n) return QADAM_ERR_STEP;
+  const float alpha = lr_t < 0.0f ? c->cfg.lr : lr_t;
+  if (!std::isfinite(alpha)) return QADAM_ERR_HYPER;
+  const ServerParams p = make_server_params(c, alpha);
+  const int grid = (int)std::min<int64_t>(c->grid_server, (int64_t)c->geo.tiles.size());
+  pick_server(c)<<<grid, kThreads, c->server_smem, c->stream>>>(p);
+  if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
+  c->launches += 1;
+  c->last_server_step = step;
+  c->workers_done = 0;
+  return QADAM_OK;
+}
+
+int qadam_step_host(qadam_ctx* c, int64_t step, const float* g_host, float* g_stage,
+                    void* out_host, float lr_t) {
+  if (!c || !g_host || !g_stage) return QADAM_ERR_NULL;
+  if (!aligned(g_stage, 16)) return QADAM_ERR_ALIGN;
+  if (step != c->last_server_step + 1 || c->workers_done != 0) return QADAM_ERR_STEP;
+  const size_t gbytes = sizeof(float) * (size_t)c->cfg.n * (size_t)c->geo.D;
+  if (!cuda_ok(cudaMemcpyAsync(g_stage, g_host, gbytes, cudaMemcpyHostToDevice, c->stream)))
+    return QADAM_ERR_CUDA;
+  int rc = qadam_worker_compress(c, step, g_stage, 0, c->cfg.n, lr_t);
+  if (rc != QADAM_OK) return rc;
+  rc = qadam_server_step(c, step, lr_t);
+  if (rc != QADAM_OK) return rc;
+  if (out_host) {
+    const bool packed = c->cfg.kx >= 0;
+    const void* src = packed ? c->buf.wcodes : static_cast<const void*>(c->buf.x);
+    const size_t bytes = packed ? c->geo.wcode_bytes : sizeof(float) * (size_t)c->geo.D;
+    if (!cuda_ok(cudaMemcpyAsync(out_host, src, bytes, cudaMemcpyDeviceToHost, c->stream)))
+      return QADAM_ERR_CUDA;
+  }
+  if (!cuda_ok(cudaStreamSynchronize(c->stream))) return QADAM_ERR_CUDA;
+  return QADAM_OK;
+}
+
+int qadam_poll_status(qadam_ctx* c, uint32_t* host_status) {
+  if (!c || !host_status) return QADAM_ERR_NULL;
+  if (!cuda_ok(cudaMemcpyAsync(host_status, c->buf.status, sizeof(uint32_t),
+                               cudaMemcpyDeviceToHost, c->stream)) ||
+      !cuda_ok(cudaStreamSynchronize(c->stream)))
+    return QADAM_ERR_CUDA;
+  return QADAM_OK;
+}
+
+int64_t qadam_launch_count(const qadam_ctx* c) { return c ? c->launches : 0; }
+
+int qadam_destroy(qadam_ctx* c) {
+  if (!c) return QADAM_ERR_NULL;
+  delete c;
+  return QADAM_OK;
+}
+
+const char* qadam_strerror(int err) {
+  switch (err) {
+    case QADAM_OK: return "ok";
+    case QADAM_ERR_NULL: return "a required pointer is NULL";
+    case QADAM_ERR_SIZE: return "invalid d, n, num_segments or segment length";
+    case QADAM_ERR_LEVEL: return "quantizer level parameter out of the supported range";
+    case QADAM_ERR_ALIGN: return "device pointer not sufficiently aligned";
+    case QADAM_ERR_WORKSPACE: return "workspace too small";
+    case QADAM_ERR_STEP: return "step out of order";
+    case QADAM_ERR_WORKER: return "worker range outside 0..n";
+    case QADAM_ERR_HYPER: return "invalid beta, theta, epsilon or step size";
+    case QADAM_ERR_CUDA: return "a CUDA call failed";
+    case QADAM_ERR_PLACEMENT: return "invalid placement";
+    default: return "unknown error";
+  }
+}
+
+int qadam_last_cuda_error(void) { return g_last_cuda_error; }
+
+}  // extern "C"

@@ -1,0 +1,230 @@
+// Device-side building blocks of the quantized-Adam step kernels (sm_100a).
+//
+// Arithmetic contract: every floating-point step of the method is one IEEE-754
+// binary32 operation with round-to-nearest-even, written with the explicit
+// __f*_rn intrinsics so that the compiler can neither contract a multiply and an
+// add into an FMA nor substitute an approximate division or square root.
+// Subnormals are kept (the library is built without flush-to-zero).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace qadam {
+
+constexpr int kAlign = 128;        // elements: segment starts, tile starts and tile lengths are multiples
+constexpr int kThreads = 256;      // threads per CTA in every kernel
+constexpr int kRows = 4;           // float4 rows per thread and tile
+constexpr int kRowElems = kThreads * 4;          // 1024 elements per CTA-wide row
+constexpr int kTileElems = kRows * kRowElems;    // 4096 elements per tile
+
+// A tile is a run of at most kTileElems padded elements inside one segment.
+struct __align__(16) Tile {
+  long long off;   // first element (padded layout), multiple of kAlign
+  int count;       // elements, multiple of kAlign
+  int seg;         // segment the run belongs to
+};
+
+// How a level index is decided and what a level is worth (Section 5.1's set G).
+enum GMode : int {
+  G_TERNARY = 0,   // {0, 1}                     (kg = 0, either grid)
+  G_FIVE = 1,      // {0, 1/2, 1}                (kg = 1, either grid)
+  G_POW2 = 2,      // {0, 2^-k, ..., 1}          (kg >= 2, geometric)
+  G_UNIFORM = 3,   // {0, 1/2^k, 2/2^k, ..., 1}  (kg >= 2, uniform)
+  G_IDENTITY = 4   // Q_g = identity
+};
+
+struct Hyper {
+  float beta, theta, eps;
+  float one_minus_beta, one_minus_theta;   // fl(1 - beta), fl(1 - theta), rounded once on the host
+};
+
+__device__ __forceinline__ float exp2i(int e) {          // 2^e, -126 <= e <= 127
+  return __int_as_float((e + 127) << 23);
+}
+
+// v_t = theta v + (1-theta) g^2 ;  m_t = beta m + (1-beta) g      (Algorithm 1 / 3)
+__device__ __forceinline__ void moments(const Hyper& h, float g, float& m, float& v) {
+  const float gg = __fmul_rn(g, g);
+  v = __fadd_rn(__fmul_rn(h.theta, v), __fmul_rn(h.one_minus_theta, gg));
+  m = __fadd_rn(__fmul_rn(h.beta, m), __fmul_rn(h.one_minus_beta, g));
+}
+
+// alpha_t m / sqrt(v + eps)      (epsilon inside the root, no bias correction)
+__device__ __forceinline__ float adam_step(const Hyper& h, float m, float v, float alpha) {
+  return __fdiv_rn(__fmul_rn(alpha, m), __fsqrt_rn(__fadd_rn(v, h.eps)));
+}
+
+// Index (0..L) of the level of G nearest to y = |u| / |u|_inf: the number of
+// midpoints between neighbouring levels that lie strictly below y, so a tie goes
+// to the level nearer zero.  y may be NaN (0/0 for an all-zero segment): every
+// comparison is then false and the index is 0.
+template <int MODE>
+__device__ __forceinline__ int level_index(float y, int k, int L) {
+  if constexpr (MODE == G_TERNARY) {
+    return y > 0.5f ? 1 : 0;
+  } else if constexpr (MODE == G_FIVE) {
+    return (y > 0.25f ? 1 : 0) + (y > 0.75f ? 1 : 0);
+  } else if constexpr (MODE == G_POW2) {
+    // levels 0, 2^-k, 2^(1-k), ..., 1: midpoints 2^(-k-1), then 3*2^(c-3-k), c = 2..L
+    float t = exp2i(-k - 1);
+    int c = y > t ? 1 : 0;
+    t = __fmul_rn(3.0f, t);
+    for (int cc = 2; cc <= L; ++cc) {
+      c += y > t ? 1 : 0;
+      t = __fmul_rn(t, 2.0f);
+    }
+    return c;
+  } else {
+    // levels c / 2^k: midpoints (c - 1/2) / 2^k.  With z = y 2^k (exact) the count
+    // of c' >= 1 with z > c' - 1/2 is ceil(z - 1/2), and z - 1/2 is exact wherever
+    // its rounding could matter (z >= 1/4).
+    const float z = __fmul_rn(y, exp2i(k));
+    int c = (int)ceilf(__fadd_rn(z, -0.5f));
+    c = c < 0 ? 0 : c;
+    return c > L ? L : c;
+  }
+}
+
+// Magnitude of level c of G (exactly representable).
+template <int MODE>
+__device__ __forceinline__ float level_value(int c, int k) {
+  if constexpr (MODE == G_TERNARY) {
+    return c ? 1.0f : 0.0f;
+  } else if constexpr (MODE == G_FIVE) {
+    return 0.5f * (float)c;
+  } else if constexpr (MODE == G_POW2) {
+    return c ? exp2i(c - 1 - k) : 0.0f;
+  } else {
+    return __fmul_rn((float)c, exp2i(-k));
+  }
+}
+
+// One coordinate of Q_g and of the error update:  given u and the segment's scale
+// s = |u|_inf, returns the code (level index + L) and writes e' = u - Q_g(u).
+template <int MODE>
+__device__ __forceinline__ unsigned quantize_grad(float u, float s, int k, int L, float& e_next) {
+  const float y = __fdiv_rn(fabsf(u), s);
+  const int c = level_index<MODE>(y, k, L);
+  const bool neg = u < 0.0f;
+  float deq = 0.0f;                                   // level 0 carries no sign
+  if (c != 0) {
+    const float mag = __fmul_rn(s, level_value<MODE>(c, k));
+    deq = neg ? -mag : mag;
+  }
+  e_next = __fsub_rn(u, deq);
+  return (unsigned)(neg ? L - c : L + c);
+}
+
+// One coordinate of Q_x (Section 5.1): nearest point of the grid c / 2^(kx+1),
+// |c| <= 2^kx, ties toward zero, clipped.  Returns the code c + 2^kx; xq is Q_x(x).
+__device__ __forceinline__ unsigned quantize_weight(float x, int kx, float& xq) {
+  const int L = 1 << kx;
+  float z = __fmul_rn(fabsf(x), exp2i(kx + 1));        // exact
+  z = fminf(z, (float)L);
+  int c = (int)ceilf(__fadd_rn(z, -0.5f));
+  c = c < 0 ? 0 : c;
+  const bool neg = x < 0.0f;
+  xq = 0.0f;
+  if (c != 0) {
+    const float mag = __fmul_rn((float)c, exp2i(-(kx + 1)));   // exact
+    xq = neg ? -mag : mag;
+  }
+  return (unsigned)(neg ? L - c : L + c);
+}
+
+// ---------------------------------------------------------------------------
+// Packing one warp-row: 32 lanes x 4 consecutive elements = 128 codes of B bits,
+// i.e. 4*B 32-bit words of the little-endian bit stream, written by lanes
+// 0..4B-1 as one coalesced store.  Every lane of the warp must call this.
+// row_dst: address of the row's first code (the row starts on a multiple of 128
+// elements, so it is 16*B-byte aligned).
+// ---------------------------------------------------------------------------
+__host__ __device__ constexpr int cgcd(int a, int b) { return b == 0 ? a : cgcd(b, a % b); }
+
+template <int B>
+__device__ __forceinline__ void pack_row_store(unsigned c0, unsigned c1, unsigned c2, unsigned c3,
+                                               void* row_dst, int lane) {
+  static_assert(B >= 2 && B <= 16, "code width");
+  if constexpr (B == 16) {
+    reinterpret_cast<uint2*>(row_dst)[lane] = make_uint2(c0 | (c1 << 16), c2 | (c3 << 16));
+  } else if constexpr (B > 8) {
+    // 4*B bits per lane (36..60): gather through shared-memory-free 64-bit shuffles
+    constexpr int F = 4 * B;                               // field width per lane
+    const unsigned long long field = (unsigned long long)c0 | ((unsigned long long)c1 << B) |
+                                     ((unsigned long long)c2 << (2 * B)) |
+                                     ((unsigned long long)c3 << (3 * B));
+    // words per row = F (<= 60): each lane produces up to two words
+#pragma unroll
+    for (int half = 0; half < 2; ++half) {
+      const int w = lane + 32 * half;
+      const int bit0 = 32 * w;
+      const int l0 = bit0 / F;
+      const int sh = bit0 - l0 * F;                        // < F
+      const unsigned long long f0 = __shfl_sync(0xffffffffu, field, l0 > 31 ? 31 : l0);
+      const unsigned long long f1 = __shfl_sync(0xffffffffu, field, l0 + 1 > 31 ? 31 : l0 + 1);
+      // bits [sh, sh+32) of the F-bit f0 followed by f1
+      unsigned long long lo = f0 >> sh;
+      const int have = F - sh;                             // bits contributed by f0 (>= 1)
+      if (have < 32) lo |= f1 << have;
+      if (w < F) reinterpret_cast<unsigned*>(row_dst)[w] = (unsigned)lo;
+    }
+  } else {
+    constexpr int F = 4 * B;                               // 8..32 bits per lane
+    constexpr int G = cgcd(32, F);
+    constexpr int J = (F - G + 32 + F - 1) / F;            // fields a 32-bit word can touch
+    const unsigned field = c0 | (c1 << B) | (c2 << (2 * B)) | (c3 << (3 * B));
+    const int bit0 = 32 * lane;
+    const int l0 = bit0 / F;
+    const int sh = bit0 - l0 * F;
+    unsigned long long acc = 0;
+#pragma unroll
+    for (int j = 0; j < J; ++j) {
+      const int src = l0 + j > 31 ? 31 : l0 + j;
+      const unsigned f = __shfl_sync(0xffffffffu, field, src);
+      acc |= (unsigned long long)f << (j * F);
+    }
+    if (lane < F) reinterpret_cast<unsigned*>(row_dst)[lane] = (unsigned)(acc >> sh);
+  }
+}
+
+// Dispatch on a run-time width.
+__device__ __forceinline__ void pack_row_store_rt(int bits, unsigned c0, unsigned c1, unsigned c2,
+                                                  unsigned c3, void* row_dst, int lane) {
+  switch (bits) {
+    case 2: pack_row_store<2>(c0, c1, c2, c3, row_dst, lane); break;
+    case 3: pack_row_store<3>(c0, c1, c2, c3, row_dst, lane); break;
+    case 4: pack_row_store<4>(c0, c1, c2, c3, row_dst, lane); break;
+    case 5: pack_row_store<5>(c0, c1, c2, c3, row_dst, lane); break;
+    case 6: pack_row_store<6>(c0, c1, c2, c3, row_dst, lane); break;
+    case 7: pack_row_store<7>(c0, c1, c2, c3, row_dst, lane); break;
+    case 8: pack_row_store<8>(c0, c1, c2, c3, row_dst, lane); break;
+    case 9: pack_row_store<9>(c0, c1, c2, c3, row_dst, lane); break;
+    case 10: pack_row_store<10>(c0, c1, c2, c3, row_dst, lane); break;
+    case 11: pack_row_store<11>(c0, c1, c2, c3, row_dst, lane); break;
+    case 12: pack_row_store<12>(c0, c1, c2, c3, row_dst, lane); break;
+    case 13: pack_row_store<13>(c0, c1, c2, c3, row_dst, lane); break;
+    case 14: pack_row_store<14>(c0, c1, c2, c3, row_dst, lane); break;
+    case 15: pack_row_store<15>(c0, c1, c2, c3, row_dst, lane); break;
+    default: pack_row_store<16>(c0, c1, c2, c3, row_dst, lane); break;
+  }
+}
+
+// The 4*bits-bit field of this lane (its 4 consecutive codes) out of a packed
+// warp-row; bits <= 8.  row_src: address of the row's first code.
+__device__ __forceinline__ unsigned unpack_row_field(const void* row_src, int bits, int lane) {
+  const int F = 4 * bits;
+  const unsigned* words = reinterpret_cast<const unsigned*>(row_src);
+  const int bit = F * lane;
+  const int w = bit >> 5;
+  const unsigned lo = __ldg(words + w);
+  const unsigned hi = __ldg(words + (w + 1 < F ? w + 1 : w));
+  const unsigned v = __funnelshift_r(lo, hi, bit & 31);
+  return F == 32 ? v : (v & ((1u << F) - 1u));
+}
+
+__device__ __forceinline__ unsigned warp_max(unsigned v) {
+  return __reduce_max_sync(0xffffffffu, v);
+}
+
+}  // namespace qadam

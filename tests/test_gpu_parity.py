@@ -1,0 +1,166 @@
+"""CUDA library vs CPU oracle, element by element, through the C interface.
+
+Packed codes, scales and packed weights must be byte-identical.  The fp32 state
+(x, m, v, e) must agree to a maximum relative error of 1e-5 (the stated bound);
+because both sides perform the same IEEE-754 binary32 operations in the same
+order it is in fact required to be bit-identical here, which is what keeps the
+codes identical over many steps."""
+import numpy as np
+import pytest
+import torch
+
+pytestmark = pytest.mark.gpu
+
+from _parity import Pair, bits_equal, rel_err  # noqa: E402
+
+import qadam_inputs as qi  # noqa: E402
+
+S_MODE, W_MODE = 0, 1
+
+
+def _rand_grads(rng, n, d, sigma=0.01):
+    return (rng.standard_normal((n, d)) * sigma).astype(np.float32)
+
+
+def _run(seg, n, kg, kx, placement, T=3, grid=0, seed=0, sigma=0.01, wresid=False, x_sigma=0.2,
+         split=False, **hyper):
+    rng = np.random.default_rng(seed)
+    d = sum(seg)
+    x1 = (rng.standard_normal(d) * x_sigma).astype(np.float32)
+    p = Pair(seg, n, kg, kx, placement, x1=x1, grid_g=grid, want_wresid=wresid, **hyper)
+    p.compare_state()                        # first broadcast Q_x(x_1)
+    for t in range(T):
+        p.step(_rand_grads(rng, n, d, sigma), split_workers=split and t % 2 == 1)
+        p.compare_state()
+    p.close()
+
+
+# ---------------------------------------------------------------- sizes: several tiles and ragged tails
+
+@pytest.mark.parametrize("d", [1, 3, 127, 128, 129, 1023, 1024, 4096, 4097, 5000, 12289, 3 * 4096 + 640])
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_flat_sizes(d, placement):
+    _run([d], 3, 0, 0, placement, T=3, seed=d)
+
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_ragged_segments(placement):
+    seg = [64, 129, 5000, 1, 4096, 9000, 7, 128, 4097]
+    _run(seg, 4, 0, 1, placement, T=4, seed=1, wresid=True, split=True)
+
+
+# ---------------------------------------------------------------- every quantizer mode
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+@pytest.mark.parametrize("kg,grid", [(-1, 0), (0, 0), (0, 1), (1, 0), (1, 1), (2, 0), (2, 1), (3, 0),
+                                     (5, 0), (14, 0), (3, 1), (4, 1), (6, 1)])
+def test_gradient_quantizer_modes(kg, grid, placement):
+    _run([3000, 200, 4100], 3, kg, 0, placement, T=3, grid=grid, seed=100 + 10 * kg + grid)
+
+
+@pytest.mark.parametrize("kx", [-1, 0, 1, 2, 3, 4, 5, 6, 7, 9, 10, 12, 13, 14])
+def test_weight_quantizer_widths(kx):
+    # x_sigma 0.4: a good share of weights falls outside [-1/2, 1/2] and is clipped
+    _run([2500, 130, 4096], 2, 0, kx, S_MODE, T=2, seed=kx + 50, wresid=True, x_sigma=0.4)
+
+
+@pytest.mark.parametrize("n", [1, 2, 5, 8, 16, 32, 33])
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_worker_counts(n, placement):
+    _run([6000, 300], n, 0, 0, placement, T=2, seed=n)
+
+
+def test_paper_hyperparameters():
+    # beta = 0.99, theta = 0.999, eps = 1e-5 (Section 5.1), moments on the workers
+    _run([5000, 64, 64, 2000], 8, 0, 6, W_MODE, T=5, seed=3, beta1=0.99, beta2=0.999, eps=1e-5)
+    _run([5000, 64, 64, 2000], 8, 1, 6, S_MODE, T=5, seed=4, beta1=0.99, beta2=0.999, eps=1e-5)
+
+
+# ---------------------------------------------------------------- degenerate and hostile values
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_zero_gradients_and_zero_segments(placement):
+    seg = [300, 4096, 50]
+    p = Pair(seg, 2, 0, 0, placement, x1=np.zeros(sum(seg), np.float32))
+    g = np.zeros((2, sum(seg)), np.float32)
+    p.step(g)                                # every scale is 0
+    p.compare_state()
+    g[0, 300:300 + 4096] = np.random.default_rng(0).standard_normal(4096).astype(np.float32)
+    p.step(g)                                # one live segment of one worker
+    p.compare_state()
+    p.close()
+
+
+@pytest.mark.parametrize("kg,grid", [(0, 0), (1, 0), (2, 0), (3, 1)])
+def test_ties_on_grid_values_and_tiny_magnitudes(kg, grid):
+    rng = np.random.default_rng(kg)
+    d = 4096 + 256
+    p = Pair([d], 2, kg, 1, S_MODE, x1=np.zeros(d, np.float32), grid_g=grid)
+    g = np.zeros((2, d), np.float32)
+    fr = np.array([1, -1, 0.5, -0.5, 0.25, 0.75, -0.75, 0.125, 0.375, 0.625, 0.875, 0.0625, 0], np.float32)
+    g[0] = rng.choice(fr, d) * np.float32(3.0)          # exact ties and on-grid values, scale 3
+    g[1] = rng.choice(fr, d) * np.float32(1e-39)        # subnormal range
+    g[0, 0], g[1, 0] = 3.0, 1e-39
+    for _ in range(3):
+        p.step(g)
+        p.compare_state()
+    p.close()
+
+
+def test_heavy_tails_and_outliers():
+    rng = np.random.default_rng(9)
+    seg = [5000, 3000]
+    p = Pair(seg, 3, 0, 0, S_MODE, x1=(rng.standard_normal(8000) * 0.02).astype(np.float32))
+    for _ in range(4):
+        g = (rng.standard_t(3, (3, 8000)) * 1e-3).astype(np.float32)
+        g[rng.integers(0, 3), rng.integers(0, 8000)] = 50.0
+        p.step(g)
+        p.compare_state()
+    p.close()
+
+
+def test_nonfinite_input_sets_status_bit():
+    import paper_2004_14180_b200 as qb
+    q = qb.QAdam([1000], 1, kg=0, kx=-1)
+    g = torch.zeros(1, q.D, device="cuda")
+    g[0, 5] = float("inf")
+    q.worker_compress(1, g)
+    assert q.poll_status() & qb.ST_NONFINITE
+    q.close()
+
+
+# ---------------------------------------------------------------- the configurations, at their sizes
+
+def _run_workload(w, steps, placement, threads=8, exact=True):
+    x1 = qi.initial_weights(w, "cpu").numpy()
+    p = Pair(w.scale_seg_len, w.n, w.kg, w.kx, placement, x1=x1,
+             beta1=w.beta1, beta2=w.beta2, eps=w.eps, lr=w.lr)
+    for t in range(1, steps + 1):
+        g = np.stack([qi.gradients(w, t, i, "cpu").numpy() for i in range(w.n)])
+        p.step(g, threads=threads)
+    p.compare_state(exact=exact)
+    ratio = p.gpu.compression_ratio()
+    p.close()
+    return ratio
+
+
+def test_config_flat20_all_steps():
+    w = qi.get_workload("flat20")
+    ratio = _run_workload(w, w.steps, S_MODE)
+    assert abs(ratio - 16.0) < 0.01                       # 32-bit -> 2-bit codes
+    _run_workload(w, w.steps, W_MODE)
+
+
+@pytest.mark.parametrize("name", ["resnet18_qg", "resnet18_qg_qx_k0", "resnet18_qg_qx_k1",
+                                  "resnet18_qg_qx_8bit"])
+def test_config_resnet18_shaped(name):
+    w = qi.get_workload(name)
+    ratio = _run_workload(w, 4, S_MODE)
+    want = 32.0 / (2 if w.kg == 0 else 3)
+    assert abs(ratio / want - 1) < 0.01                   # per-tensor scales and padding cost < 1 %
+
+
+def test_config_resnet18_shaped_paper_placement_and_single_scale():
+    w = qi.get_workload("resnet18_qg_qx_k0")
+    _run_workload(w, 3, W_MODE)
+    _run_workload(w.with_(per_tensor_scale=False), 3, S_MODE)
