@@ -173,6 +173,23 @@ int qadam_step_host(qadam_ctx* ctx, int64_t step, const float* g_host, float* g_
 /* Waits for the context's stream, then copies the status word to *host_status. */
 int qadam_poll_status(qadam_ctx* ctx, uint32_t* host_status);
 
+/* Instrumentation (no counterpart in the paper).  While enabled, every kernel the
+ * context launches is bracketed by CUDA events on the context's stream.
+ * qadam_profile_read waits for the stream, adds the elapsed device time of the
+ * launches since the last read to ms[kind] and their number to launches[kind]
+ * (host arrays of QADAM_NUM_KERNELS entries, which the caller zeroes), and
+ * forgets them. */
+enum {
+  QADAM_K_ABSMAX = 0,      /* worker phase 1: form u, max|u| per (worker, segment)  */
+  QADAM_K_QUANTIZE = 1,    /* worker phase 2: level indices, packing, e <- u - Q_g(u) */
+  QADAM_K_IDENTITY = 2,    /* worker with Q_g = identity                              */
+  QADAM_K_SERVER = 3,      /* fused server pass                                       */
+  QADAM_K_BROADCAST = 4,   /* stand-alone Q_x(x_1)                                    */
+  QADAM_NUM_KERNELS = 5
+};
+int qadam_profile_enable(qadam_ctx* ctx, int enable);
+int qadam_profile_read(qadam_ctx* ctx, double* ms, int64_t* launches);
+
 /* Number of kernels this context has launched since it was created. */
 int64_t qadam_launch_count(const qadam_ctx* ctx);
 

@@ -23,7 +23,10 @@ exported_symbols = (
     "qadam_query_sizes", "qadam_grad_code_bits", "qadam_weight_code_bits", "qadam_create",
     "qadam_worker_compress", "qadam_server_step", "qadam_step_host", "qadam_poll_status",
     "qadam_launch_count", "qadam_destroy", "qadam_strerror", "qadam_last_cuda_error",
+    "qadam_profile_enable", "qadam_profile_read",
 )
+
+KERNEL_NAMES = ("absmax", "quantize", "identity", "server", "broadcast")
 
 
 class QAdamError(RuntimeError):
@@ -89,6 +92,10 @@ def load_library():
     L.qadam_step_host.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_void_p, C.c_void_p, C.c_float]
     L.qadam_poll_status.restype = C.c_int
     L.qadam_poll_status.argtypes = [C.c_void_p, C.POINTER(C.c_uint32)]
+    L.qadam_profile_enable.restype = C.c_int
+    L.qadam_profile_enable.argtypes = [C.c_void_p, C.c_int]
+    L.qadam_profile_read.restype = C.c_int
+    L.qadam_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     L.qadam_launch_count.restype = C.c_int64
     L.qadam_launch_count.argtypes = [C.c_void_p]
     L.qadam_destroy.restype = C.c_int
@@ -158,6 +165,18 @@ def qadam_poll_status(ctx: int) -> int:
     st = C.c_uint32()
     _check(load_library().qadam_poll_status(ctx, C.byref(st)), "qadam_poll_status")
     return st.value
+
+
+def qadam_profile_enable(ctx: int, enable: bool) -> None:
+    _check(load_library().qadam_profile_enable(ctx, int(bool(enable))), "qadam_profile_enable")
+
+
+def qadam_profile_read(ctx: int):
+    """-> {kernel name: (total ms, launches)} since the last read."""
+    n = len(KERNEL_NAMES)
+    ms, cnt = (C.c_double * n)(), (C.c_int64 * n)()
+    _check(load_library().qadam_profile_read(ctx, ms, cnt), "qadam_profile_read")
+    return {KERNEL_NAMES[i]: (ms[i], cnt[i]) for i in range(n)}
 
 
 def qadam_launch_count(ctx: int) -> int:
@@ -270,6 +289,12 @@ class QAdam:
         assert g_stage.is_cuda and g_stage.numel() == self.n * self.D
         qadam_step_host(self.ctx, step, g_host.data_ptr(), g_stage.data_ptr(),
                         out_host.data_ptr() if out_host is not None else None, lr)
+
+    def profile(self, enable: bool) -> None:
+        qadam_profile_enable(self.ctx, enable)
+
+    def profile_read(self):
+        return qadam_profile_read(self.ctx)
 
     def poll_status(self) -> int:
         return qadam_poll_status(self.ctx)

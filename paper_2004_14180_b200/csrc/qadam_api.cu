@@ -129,6 +129,11 @@ struct qadam_ctx {
   int64_t launches;
   int grid_absmax, grid_quant, grid_ident, grid_server, grid_bcast;
   size_t server_smem;
+  // instrumentation: event pairs of the launches since the last read
+  bool profiling = false;
+  struct Timed { int kind; cudaEvent_t start, stop; };
+  std::vector<Timed> timed;
+  std::vector<cudaEvent_t> spare_events;
 };
 
 namespace {
@@ -174,6 +179,37 @@ ServerKernel pick_server(const qadam_ctx* c) {
     default:         return s ? server_step_kernel<true, G_IDENTITY> : server_step_kernel<false, G_IDENTITY>;
   }
 }
+
+cudaEvent_t take_event(qadam_ctx* c) {
+  if (!c->spare_events.empty()) {
+    cudaEvent_t e = c->spare_events.back();
+    c->spare_events.pop_back();
+    return e;
+  }
+  cudaEvent_t e = nullptr;
+  cuda_ok(cudaEventCreate(&e));
+  return e;
+}
+
+// Brackets one kernel launch with events while profiling is on.
+struct LaunchTimer {
+  qadam_ctx* c;
+  qadam_ctx::Timed t;
+  LaunchTimer(qadam_ctx* ctx, int kind) : c(ctx) {
+    t.kind = kind; t.start = t.stop = nullptr;
+    if (c->profiling) {
+      t.start = take_event(c);
+      t.stop = take_event(c);
+      if (t.start) cudaEventRecord(t.start, c->stream);
+    }
+  }
+  ~LaunchTimer() {
+    if (c->profiling && t.start && t.stop) {
+      cudaEventRecord(t.stop, c->stream);
+      c->timed.push_back(t);
+    }
+  }
+};
 
 ServerParams make_server_params(const qadam_ctx* c, float alpha) {
   ServerParams p;
@@ -290,7 +326,10 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
   if (quant_x) {
     const ServerParams p = make_server_params(c, 0.0f);
     const int grid = (int)std::min<int64_t>(c->grid_bcast, (int64_t)c->geo.tiles.size());
-    weight_broadcast_kernel<<<grid, kThreads, 0, c->stream>>>(p);
+    {
+      LaunchTimer lt(c, QADAM_K_BROADCAST);
+      weight_broadcast_kernel<<<grid, kThreads, 0, c->stream>>>(p);
+    }
     if (!cuda_ok(cudaGetLastError())) { delete c; return QADAM_ERR_CUDA; }
     c->launches++;
   }
@@ -327,7 +366,10 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
 
   if (c->geo.gmode == G_IDENTITY) {
     const int grid = (int)std::min<int64_t>(c->grid_ident, p.total_tiles);
-    pick_identity(c)<<<grid, kThreads, 0, c->stream>>>(p);
+    {
+      LaunchTimer lt(c, QADAM_K_IDENTITY);
+      pick_identity(c)<<<grid, kThreads, 0, c->stream>>>(p);
+    }
     if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
     c->launches += 1;
   } else {
@@ -335,10 +377,16 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
                                  sizeof(unsigned) * (size_t)worker_count * p.S, c->stream)))
       return QADAM_ERR_CUDA;
     int grid = (int)std::min<int64_t>(c->grid_absmax, p.total_tiles);
-    pick_absmax(c)<<<grid, kThreads, 0, c->stream>>>(p);
+    {
+      LaunchTimer lt(c, QADAM_K_ABSMAX);
+      pick_absmax(c)<<<grid, kThreads, 0, c->stream>>>(p);
+    }
     if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
     grid = (int)std::min<int64_t>(c->grid_quant, p.total_tiles);
-    pick_quantize(c)<<<grid, kThreads, 0, c->stream>>>(p);
+    {
+      LaunchTimer lt(c, QADAM_K_QUANTIZE);
+      pick_quantize(c)<<<grid, kThreads, 0, c->stream>>>(p);
+    }
     if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
     c->launches += 2;
   }
@@ -353,7 +401,10 @@ int qadam_server_step(qadam_ctx* c, int64_t step, float lr_t) {
   if (!std::isfinite(alpha)) return QADAM_ERR_HYPER;
   const ServerParams p = make_server_params(c, alpha);
   const int grid = (int)std::min<int64_t>(c->grid_server, (int64_t)c->geo.tiles.size());
-  pick_server(c)<<<grid, kThreads, c->server_smem, c->stream>>>(p);
+  {
+    LaunchTimer lt(c, QADAM_K_SERVER);
+    pick_server(c)<<<grid, kThreads, c->server_smem, c->stream>>>(p);
+  }
   if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
   c->launches += 1;
   c->last_server_step = step;
@@ -393,10 +444,37 @@ int qadam_poll_status(qadam_ctx* c, uint32_t* host_status) {
   return QADAM_OK;
 }
 
+int qadam_profile_enable(qadam_ctx* c, int enable) {
+  if (!c) return QADAM_ERR_NULL;
+  c->profiling = enable != 0;
+  return QADAM_OK;
+}
+
+int qadam_profile_read(qadam_ctx* c, double* ms, int64_t* launches) {
+  if (!c || !ms || !launches) return QADAM_ERR_NULL;
+  if (!cuda_ok(cudaStreamSynchronize(c->stream))) return QADAM_ERR_CUDA;
+  for (const qadam_ctx::Timed& t : c->timed) {
+    float el = 0.0f;
+    if (cuda_ok(cudaEventElapsedTime(&el, t.start, t.stop))) {
+      ms[t.kind] += el;
+      launches[t.kind] += 1;
+    }
+    c->spare_events.push_back(t.start);
+    c->spare_events.push_back(t.stop);
+  }
+  c->timed.clear();
+  return QADAM_OK;
+}
+
 int64_t qadam_launch_count(const qadam_ctx* c) { return c ? c->launches : 0; }
 
 int qadam_destroy(qadam_ctx* c) {
   if (!c) return QADAM_ERR_NULL;
+  for (const qadam_ctx::Timed& t : c->timed) {
+    cudaEventDestroy(t.start);
+    cudaEventDestroy(t.stop);
+  }
+  for (cudaEvent_t e : c->spare_events) cudaEventDestroy(e);
   delete c;
   return QADAM_OK;
 }
