@@ -12,6 +12,9 @@
 #include <vector>
 
 #include "qadam_kernels.cuh"
+#include "qadam_server_pipe.cuh"
+
+#include <cstdlib>
 
 using namespace qadam;
 
@@ -129,6 +132,9 @@ struct qadam_ctx {
   int64_t launches;
   int grid_absmax, grid_quant, grid_ident, grid_server, grid_bcast;
   size_t server_smem;
+  // persistent pipelined server pass (ternary codes): stages > 0 when in use
+  int pipe_stages = 0;
+  size_t pipe_smem = 0;
   // instrumentation: event pairs of the launches since the last read
   bool profiling = false;
   struct Timed { int kind; cudaEvent_t start, stop; };
@@ -228,6 +234,8 @@ ServerParams make_server_params(const qadam_ctx* c, float alpha) {
   p.kx = c->cfg.kx; p.xbits = c->geo.xbits;
   p.alpha = alpha;
   p.nf = (float)c->cfg.n;
+  p.inv_nf = 1.0f / (float)c->cfg.n;
+  p.status = c->buf.status;
   p.h = c->h;
   return p;
 }
@@ -305,6 +313,28 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
   if (c->server_smem > 48 * 1024 &&
       !cuda_ok(cudaFuncSetAttribute(sk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->server_smem))) {
     delete c; return QADAM_ERR_CUDA;
+  }
+  // The pipelined server pass needs ternary codes, at most kPipeMaxWorkers streams and room
+  // for at least two stages in shared memory; otherwise the plain grid-stride kernel runs.
+  {
+    int max_smem = 0;
+    if (!cuda_ok(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev))) {
+      delete c; return QADAM_ERR_CUDA;
+    }
+    const bool sm_mom = cfg->placement == QADAM_PLACE_SERVER;
+    const size_t sb = pipe_stage_bytes(cfg->n, sm_mom);
+    const char* env = std::getenv("QADAM_SERVER_KERNEL");
+    const bool want_plain = env && std::strcmp(env, "plain") == 0;
+    int stages = (int)(((size_t)max_smem - 256) / sb);
+    stages = std::min(stages, kPipeMaxStages);
+    if (!want_plain && c->geo.gmode == G_TERNARY && cfg->n <= kPipeMaxWorkers && stages >= 2) {
+      c->pipe_stages = stages;
+      c->pipe_smem = 256 + (size_t)stages * sb;
+      const cudaError_t e = sm_mom
+          ? cudaFuncSetAttribute(server_pipe_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pipe_smem)
+          : cudaFuncSetAttribute(server_pipe_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pipe_smem);
+      if (!cuda_ok(e)) { delete c; return QADAM_ERR_CUDA; }
+    }
   }
   c->grid_absmax = resident_grid(pick_absmax(c), 0, c->sm_count);
   c->grid_quant = resident_grid(pick_quantize(c), 0, c->sm_count);
@@ -403,7 +433,17 @@ int qadam_server_step(qadam_ctx* c, int64_t step, float lr_t) {
   const int grid = (int)std::min<int64_t>(c->grid_server, (int64_t)c->geo.tiles.size());
   {
     LaunchTimer lt(c, QADAM_K_SERVER);
-    pick_server(c)<<<grid, kThreads, c->server_smem, c->stream>>>(p);
+    if (c->pipe_stages > 0) {
+      const int n = c->cfg.n;
+      const int inv_exact = (n & (n - 1)) == 0 ? 1 : 0;
+      const int pgrid = (int)std::min<int64_t>(c->sm_count, 2 * (int64_t)c->geo.tiles.size());
+      if (c->cfg.placement == QADAM_PLACE_SERVER)
+        server_pipe_kernel<true><<<pgrid, kPipeThreads, c->pipe_smem, c->stream>>>(p, c->pipe_stages, inv_exact);
+      else
+        server_pipe_kernel<false><<<pgrid, kPipeThreads, c->pipe_smem, c->stream>>>(p, c->pipe_stages, inv_exact);
+    } else {
+      pick_server(c)<<<grid, kThreads, c->server_smem, c->stream>>>(p);
+    }
   }
   if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
   c->launches += 1;

@@ -51,6 +51,8 @@ struct ServerParams {
   int kx, xbits;         // weight level parameter (-1: none) / code width
   float alpha;
   float nf;              // (float)n
+  float inv_nf;          // 1/n, exact when n is a power of two
+  unsigned* status;
   Hyper h;
 };
 

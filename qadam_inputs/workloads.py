@@ -92,6 +92,11 @@ def get_workload(name: str, n: Optional[int] = None) -> Workload:
         seg, fan, gam = _flat(1 << 28)
         w = Workload("flat28", seg, fan, gam, n=16, steps=20, grad="mixture",
                      w0="gauss:0.05", kg=0, kx=0)
+    elif name.startswith("flat") and name[4:].isdigit() and 10 <= int(name[4:]) <= 30:
+        # the flat28 recipe at another power-of-two length (profiling and sampling)
+        seg, fan, gam = _flat(1 << int(name[4:]))
+        w = Workload(name, seg, fan, gam, n=16, steps=20, grad="mixture",
+                     w0="gauss:0.05", kg=0, kx=0)
     else:
         raise KeyError(f"unknown workload {name!r}; known: {WORKLOAD_NAMES}")
     if n is not None:
