@@ -51,7 +51,8 @@ int grad_levels(int kg, int grid) {
 struct Geometry {
   std::vector<int64_t> seg_len, seg_off;
   int64_t D = 0;
-  std::vector<Tile> tiles;
+  std::vector<Tile> tiles;        // runs of at most kTileElems
+  std::vector<Tile> ptiles;       // the same vector cut into runs of at most kPipeTile
   int gbits = 0, xbits = 0, L = 0;
   GMode gmode = G_TERNARY;
   size_t gcode_bytes = 0, wcode_bytes = 0, workspace_bytes = 0;
@@ -92,6 +93,7 @@ int build_geometry(const qadam_config* c, Geometry* g) {
   g->D = off;
   if (g->D / kAlign > (int64_t)1 << 30) return QADAM_ERR_SIZE;
   g->tiles.clear();
+  g->ptiles.clear();
   for (int s = 0; s < S; ++s) {
     const int64_t plen = round_up64(g->seg_len[s], kAlign);
     for (int64_t o = 0; o < plen; o += kTileElems) {
@@ -100,6 +102,13 @@ int build_geometry(const qadam_config* c, Geometry* g) {
       t.count = (int)std::min<int64_t>(kTileElems, plen - o);
       t.seg = s;
       g->tiles.push_back(t);
+    }
+    for (int64_t o = 0; o < plen; o += kPipeTile) {
+      Tile t;
+      t.off = g->seg_off[s] + o;
+      t.count = (int)std::min<int64_t>(kPipeTile, plen - o);
+      t.seg = s;
+      g->ptiles.push_back(t);
     }
   }
   if (c->kg < 0) {
@@ -113,7 +122,8 @@ int build_geometry(const qadam_config* c, Geometry* g) {
   g->xbits = c->kx < 0 ? 0 : c->kx + 2;
   g->gcode_bytes = (size_t)(g->D * g->gbits / 8);
   g->wcode_bytes = (size_t)(g->D * g->xbits / 8);
-  g->workspace_bytes = (size_t)round_up64((int64_t)g->tiles.size() * sizeof(Tile), 256) + 256;
+  g->workspace_bytes = (size_t)round_up64((int64_t)g->tiles.size() * sizeof(Tile), 256) +
+                       (size_t)round_up64((int64_t)g->ptiles.size() * sizeof(Tile), 256) + 256;
   return QADAM_OK;
 }
 
@@ -126,6 +136,7 @@ struct qadam_ctx {
   Hyper h;
   cudaStream_t stream;
   Tile* d_tiles;
+  Tile* d_ptiles;
   int sm_count;
   int64_t last_server_step;     // steps completed by the server
   int64_t workers_done;         // workers compressed for step last_server_step + 1
@@ -184,6 +195,23 @@ ServerKernel pick_server(const qadam_ctx* c) {
     case G_UNIFORM:  return s ? server_step_kernel<true, G_UNIFORM>  : server_step_kernel<false, G_UNIFORM>;
     default:         return s ? server_step_kernel<true, G_IDENTITY> : server_step_kernel<false, G_IDENTITY>;
   }
+}
+
+using PipeKernel = void (*)(const ServerParams, const Tile*, int, int, int);
+
+template <bool SM>
+PipeKernel pick_pipe_n(int n) {
+  switch (n) {
+    case 4: return server_pipe_kernel<SM, 4>;
+    case 8: return server_pipe_kernel<SM, 8>;
+    case 16: return server_pipe_kernel<SM, 16>;
+    case 32: return server_pipe_kernel<SM, 32>;
+    default: return server_pipe_kernel<SM, 0>;
+  }
+}
+
+PipeKernel pick_pipe(const qadam_ctx* c) {
+  return c->cfg.placement == QADAM_PLACE_SERVER ? pick_pipe_n<true>(c->cfg.n) : pick_pipe_n<false>(c->cfg.n);
 }
 
 cudaEvent_t take_event(qadam_ctx* c) {
@@ -299,6 +327,8 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
   c->workers_done = 0;
   c->launches = 0;
   c->d_tiles = static_cast<Tile*>(b->workspace);
+  c->d_ptiles = reinterpret_cast<Tile*>(static_cast<unsigned char*>(b->workspace) +
+                                        round_up64((int64_t)c->geo.tiles.size() * sizeof(Tile), 256));
 
   int dev = 0;
   if (!cuda_ok(cudaGetDevice(&dev)) ||
@@ -330,10 +360,10 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
     if (!want_plain && c->geo.gmode == G_TERNARY && cfg->n <= kPipeMaxWorkers && stages >= 2) {
       c->pipe_stages = stages;
       c->pipe_smem = 256 + (size_t)stages * sb;
-      const cudaError_t e = sm_mom
-          ? cudaFuncSetAttribute(server_pipe_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pipe_smem)
-          : cudaFuncSetAttribute(server_pipe_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pipe_smem);
-      if (!cuda_ok(e)) { delete c; return QADAM_ERR_CUDA; }
+      if (!cuda_ok(cudaFuncSetAttribute(pick_pipe(c), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                        (int)c->pipe_smem))) {
+        delete c; return QADAM_ERR_CUDA;
+      }
     }
   }
   c->grid_absmax = resident_grid(pick_absmax(c), 0, c->sm_count);
@@ -348,6 +378,8 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
 
   // tables and status: synchronous, so the host vector may go away
   if (!cuda_ok(cudaMemcpyAsync(c->d_tiles, c->geo.tiles.data(), c->geo.tiles.size() * sizeof(Tile),
+                               cudaMemcpyHostToDevice, c->stream)) ||
+      !cuda_ok(cudaMemcpyAsync(c->d_ptiles, c->geo.ptiles.data(), c->geo.ptiles.size() * sizeof(Tile),
                                cudaMemcpyHostToDevice, c->stream)) ||
       !cuda_ok(cudaMemsetAsync(b->status, 0, sizeof(uint32_t), c->stream)) ||
       !cuda_ok(cudaStreamSynchronize(c->stream))) {
@@ -436,11 +468,9 @@ int qadam_server_step(qadam_ctx* c, int64_t step, float lr_t) {
     if (c->pipe_stages > 0) {
       const int n = c->cfg.n;
       const int inv_exact = (n & (n - 1)) == 0 ? 1 : 0;
-      const int pgrid = (int)std::min<int64_t>(c->sm_count, 2 * (int64_t)c->geo.tiles.size());
-      if (c->cfg.placement == QADAM_PLACE_SERVER)
-        server_pipe_kernel<true><<<pgrid, kPipeThreads, c->pipe_smem, c->stream>>>(p, c->pipe_stages, inv_exact);
-      else
-        server_pipe_kernel<false><<<pgrid, kPipeThreads, c->pipe_smem, c->stream>>>(p, c->pipe_stages, inv_exact);
+      const int np = (int)c->geo.ptiles.size();
+      const int pgrid = std::min(c->sm_count, np);
+      pick_pipe(c)<<<pgrid, kPipeThreads, c->pipe_smem, c->stream>>>(p, c->d_ptiles, np, c->pipe_stages, inv_exact);
     } else {
       pick_server(c)<<<grid, kThreads, c->server_smem, c->stream>>>(p);
     }

@@ -51,8 +51,16 @@ __device__ __forceinline__ void moments(const Hyper& h, float g, float& m, float
 }
 
 // alpha_t m / sqrt(v + eps)      (epsilon inside the root, no bias correction)
+// A zero numerator is frequent (a coordinate whose decoded updates have all been
+// level 0 keeps m = 0 exactly) and would send the IEEE division down its slow
+// special-case path; +-0 / den = +-0 for the positive den here, so the numerator is
+// returned as it is and the divider is fed a harmless 1 in its place.
 __device__ __forceinline__ float adam_step(const Hyper& h, float m, float v, float alpha) {
-  return __fdiv_rn(__fmul_rn(alpha, m), __fsqrt_rn(__fadd_rn(v, h.eps)));
+  const float num = __fmul_rn(alpha, m);
+  const float den = __fsqrt_rn(__fadd_rn(v, h.eps));
+  const bool zero = num == 0.0f;
+  const float q = __fdiv_rn(zero ? 1.0f : num, den);
+  return zero ? num : q;
 }
 
 // Index (0..L) of the level of G nearest to y = |u| / |u|_inf: the number of
@@ -119,6 +127,13 @@ __device__ __forceinline__ unsigned quantize_grad(float u, float s, int k, int L
 // One coordinate of Q_x (Section 5.1): nearest point of the grid c / 2^(kx+1),
 // |c| <= 2^kx, ties toward zero, clipped.  Returns the code c + 2^kx; xq is Q_x(x).
 __device__ __forceinline__ unsigned quantize_weight(float x, int kx, float& xq) {
+  if (kx == 0) {
+    // grid {-1/2, 0, 1/2}: the single midpoint is 1/4 (z = 2|x| > 1/2), ties toward zero
+    const bool far = fabsf(x) > 0.25f;
+    const bool neg = x < 0.0f;
+    xq = far ? (neg ? -0.5f : 0.5f) : 0.0f;
+    return far ? (neg ? 0u : 2u) : 1u;
+  }
   const int L = 1 << kx;
   float z = __fmul_rn(fabsf(x), exp2i(kx + 1));        // exact
   z = fminf(z, (float)L);
@@ -221,6 +236,37 @@ __device__ __forceinline__ unsigned unpack_row_field(const void* row_src, int bi
   const unsigned hi = __ldg(words + (w + 1 < F ? w + 1 : w));
   const unsigned v = __funnelshift_r(lo, hi, bit & 31);
   return F == 32 ? v : (v & ((1u << F) - 1u));
+}
+
+// Packed binary32 arithmetic (two independent lanes per instruction, sm_100).
+// Each lane rounds exactly like the scalar operation.  Caution: unlike the scalar
+// forms, a packed multiply whose result feeds a packed add IS fused into a packed
+// fused multiply-add by the assembler, explicit rounding mode or not (measured on
+// sm_100a, CUDA 12.9): never feed mul2_rn into add2_rn where both roundings matter.
+__device__ __forceinline__ unsigned long long pack_f2(float2 a) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(a.x), "f"(a.y));
+  return r;
+}
+__device__ __forceinline__ float2 unpack_f2(unsigned long long r) {
+  float2 a;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(a.x), "=f"(a.y) : "l"(r));
+  return a;
+}
+__device__ __forceinline__ float2 add2_rn(float2 a, float2 b) {
+  unsigned long long r;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(pack_f2(a)), "l"(pack_f2(b)));
+  return unpack_f2(r);
+}
+__device__ __forceinline__ float2 mul2_rn(float2 a, float2 b) {
+  unsigned long long r;
+  asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(r) : "l"(pack_f2(a)), "l"(pack_f2(b)));
+  return unpack_f2(r);
+}
+__device__ __forceinline__ float2 fma2_rn(float2 a, float2 b, float2 c) {
+  unsigned long long r;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(r) : "l"(pack_f2(a)), "l"(pack_f2(b)), "l"(pack_f2(c)));
+  return unpack_f2(r);
 }
 
 __device__ __forceinline__ unsigned warp_max(unsigned v) {

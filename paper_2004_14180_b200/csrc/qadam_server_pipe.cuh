@@ -3,9 +3,9 @@
 // One CTA per SM loops over 2048-element tiles.  A producer warp brings each
 // tile's inputs (x, m, v and the n workers' 512-byte code runs) into a ring of
 // shared-memory stages with bulk asynchronous copies that complete on an
-// mbarrier; sixteen consumer warps decode, average and update in place in shared
-// memory and write the packed broadcast; a storer warp sends the updated x, m, v
-// back with bulk stores and frees the stage.  Global-memory latency is covered by
+// mbarrier; two groups of eight consumer warps take alternate tiles, decode,
+// average and update in place in shared memory and write the packed broadcast; a
+// storer warp sends the updated x, m, v back with bulk stores and frees the stage.  Global-memory latency is covered by
 // the copies in flight (stages x tile bytes per SM), not by occupancy, so the
 // consumers keep their registers for arithmetic.
 //
@@ -20,6 +20,7 @@ namespace qadam {
 
 constexpr int kPipeTile = 2048;                 // elements per pipeline tile
 constexpr int kPipeConsumers = 512;             // 16 warps, 4 elements per thread
+constexpr int kPipeGroupThreads = 256;          // two consumer groups take alternate tiles
 constexpr int kPipeThreads = kPipeConsumers + 64;   // + producer warp + storer warp
 constexpr int kPipeMaxWorkers = 64;
 constexpr int kPipeMaxStages = 8;
@@ -90,35 +91,103 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsig
 }
 
 struct PipeSmem {
-  unsigned long long full[kPipeMaxStages];      // producer -> consumers (bytes landed, scales written)
+  unsigned long long full[kPipeMaxStages];      // producer -> consumers (bytes landed, header and scales written)
   unsigned long long computed[kPipeMaxStages];  // consumers -> storer
   unsigned long long empty[kPipeMaxStages];     // storer -> producer
   int abort_flag;
 };
 
-// Bytes of one stage: x, m, v tiles, the code runs of n workers, n scales.
+// A stage: [header 128 B][x tile][m tile][v tile][n code runs of 512 B][n scales, each stored twice]
+struct StageHeader {
+  long long off;   // first element of the tile
+  int count;       // its length (multiple of 128, at most kPipeTile)
+  int pad;
+};
+constexpr int kStageHeaderBytes = 128;
+
 __host__ __device__ inline size_t pipe_stage_bytes(int n, bool server_moments) {
   const size_t state = (server_moments ? 3 : 1) * (size_t)kPipeTile * sizeof(float);
   const size_t codes = (size_t)n * (kPipeTile / 4);
-  const size_t scales = ((size_t)n * sizeof(float) + 127) / 128 * 128;
-  return state + codes + scales;
+  const size_t scales = ((size_t)n * 2 * sizeof(float) + 127) / 128 * 128;
+  return kStageHeaderBytes + state + codes + scales;
 }
 
-template <bool SERVER_MOMENTS>
+// v, m updates of Algorithm 1 / 3 on two coordinates at once.  Only the products
+// are packed: the assembler fuses a packed multiply that feeds a packed add into one
+// fused multiply-add even when both carry an explicit rounding mode (measured), which
+// would drop a rounding; the scalar add with explicit rounding is never fused.
+__device__ __forceinline__ void moments2(const Hyper& h, float2 g, float2& m, float2& v) {
+  const float2 gg = mul2_rn(g, g);
+  const float2 tv = mul2_rn(make_float2(h.theta, h.theta), v);
+  const float2 og = mul2_rn(make_float2(h.one_minus_theta, h.one_minus_theta), gg);
+  const float2 bm = mul2_rn(make_float2(h.beta, h.beta), m);
+  const float2 ob = mul2_rn(make_float2(h.one_minus_beta, h.one_minus_beta), g);
+  v = make_float2(__fadd_rn(tv.x, og.x), __fadd_rn(tv.y, og.y));
+  m = make_float2(__fadd_rn(bm.x, ob.x), __fadd_rn(bm.y, ob.y));
+}
+
+// One worker's contribution to the 8 running sums of a consumer thread.
+//   sc    (scale, scale) of the worker
+//   b0,b1 the thread's code bytes of the tile's two rows (4 two-bit codes each)
+// A code c sits in mantissa bits [2c', 2c'+2) of a float whose exponent gives that
+// position the weight 1 (value 2^E + code); subtracting 2^E + 1 leaves the level
+// index (-1, 0, 1) as a float, and fma(index, scale, sum) = fl(sum + index*scale)
+// rounds exactly like adding the decoded value because the product is exact.
+// mg[c']: the bit pattern of 2^(23 - 2c'), held in registers that the compiler
+// cannot see through, so that (byte & mask) | pattern is one three-input logic
+// operation with a single immediate instead of two operations.
+template <unsigned MASK_LO, unsigned MASK_HI>
+__device__ __forceinline__ float2 code_pair_minus_bias(unsigned b, unsigned mg_lo, unsigned mg_hi,
+                                                       float2 k) {
+  // {lo, hi} = {(b & MASK_LO) | mg_lo, (b & MASK_HI) | mg_hi}, each one three-input
+  // logic operation (truth table 0xEA = (a & b) | c), built straight into the two
+  // halves of the packed operand; then the packed subtraction of 2^E + 1.
+  unsigned long long r;
+  asm("{\n\t.reg .b32 lo, hi;\n\t.reg .b64 t;\n\t"
+      "lop3.b32 lo, %1, %2, %3, 0xEA;\n\t"
+      "lop3.b32 hi, %1, %4, %5, 0xEA;\n\t"
+      "mov.b64 t, {lo, hi};\n\t"
+      "add.rn.f32x2 %0, t, %6;\n\t}"
+      : "=l"(r)
+      : "r"(b), "n"(MASK_LO), "r"(mg_lo), "n"(MASK_HI), "r"(mg_hi), "l"(pack_f2(k)));
+  return unpack_f2(r);
+}
+
+__device__ __forceinline__ void decode_accumulate(float2 sc, unsigned b0, unsigned b1, float2 k01,
+                                                  float2 k23, const unsigned (&mg)[4], float2 (&a)[4]) {
+  a[0] = fma2_rn(code_pair_minus_bias<0x03u, 0x0cu>(b0, mg[0], mg[1], k01), sc, a[0]);
+  a[1] = fma2_rn(code_pair_minus_bias<0x30u, 0xc0u>(b0, mg[2], mg[3], k23), sc, a[1]);
+  a[2] = fma2_rn(code_pair_minus_bias<0x03u, 0x0cu>(b1, mg[0], mg[1], k01), sc, a[2]);
+  a[3] = fma2_rn(code_pair_minus_bias<0x30u, 0xc0u>(b1, mg[2], mg[3], k23), sc, a[3]);
+}
+
+__device__ __forceinline__ unsigned opaque_u32(unsigned v) {
+  unsigned r;
+  asm volatile("mov.u32 %0, %1;" : "=r"(r) : "r"(v));
+  return r;
+}
+
+// NW > 0: the worker count, known at compile time (the decode loop is unrolled and
+// every shared-memory offset is an immediate).  NW = 0: p.n workers, run-time loop.
+template <bool SERVER_MOMENTS, int NW>
 __global__ void __launch_bounds__(kPipeThreads, 1)
-server_pipe_kernel(const ServerParams p, const int stages, const int inv_n_exact) {
+server_pipe_kernel(const ServerParams p, const Tile* __restrict__ ptiles, const int num_ptiles,
+                   const int stages, const int inv_n_exact) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   PipeSmem* ps = reinterpret_cast<PipeSmem*>(smem_raw);
   unsigned char* stage_base = smem_raw + 256;
-  const size_t stage_bytes = pipe_stage_bytes(p.n, SERVER_MOMENTS);
+  const int n = NW > 0 ? NW : p.n;
+  const unsigned stage_bytes = (unsigned)pipe_stage_bytes(n, SERVER_MOMENTS);
   constexpr int kState = SERVER_MOMENTS ? 3 : 1;
+  constexpr unsigned kCodesOff = kStageHeaderBytes + kState * kPipeTile * 4;
+  const unsigned scales_off = kCodesOff + (unsigned)n * (kPipeTile / 4);
   const int tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
 
   if (tid == 0) {
     for (int s = 0; s < stages; ++s) {
       mbar_init(&ps->full[s], 1);
-      mbar_init(&ps->computed[s], kPipeConsumers / 32);
+      mbar_init(&ps->computed[s], kPipeGroupThreads / 32);
       mbar_init(&ps->empty[s], 1);
     }
     ps->abort_flag = 0;
@@ -126,168 +195,194 @@ server_pipe_kernel(const ServerParams p, const int stages, const int inv_n_exact
   }
   __syncthreads();
 
-  // Tiles of this CTA: halves h = blockIdx.x, blockIdx.x + gridDim.x, ... of the 4096-element table.
-  const long long num_halves = 2LL * p.tiles_per_worker;
   volatile int* abort_flag = &ps->abort_flag;
-
-  auto stage_ptr = [&](int s) { return stage_base + (size_t)s * stage_bytes; };
-  auto half_tile = [&](long long h, long long& off, int& count, int& seg) {
-    const Tile t = p.tiles[(int)(h >> 1)];
-    const int skip = (int)(h & 1) * kPipeTile;
-    off = t.off + skip;
-    count = t.count - skip;
-    count = count > kPipeTile ? kPipeTile : count;
-    seg = t.seg;
-  };
+  // tiles of this CTA: blockIdx.x, blockIdx.x + gridDim.x, ...
+  const int my_tiles = (int)blockIdx.x < num_ptiles
+                           ? (num_ptiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
 
   if (warp == kPipeConsumers / 32) {
     // ------------------------------------------------------------------ producer
     int cur_seg = -1;
     float sc0 = 0.0f, sc1 = 0.0f;                       // scales of workers lane, lane + 32
-    long long j = 0;
-    for (long long h = blockIdx.x; h < num_halves; h += gridDim.x) {
-      long long off; int count, seg;
-      half_tile(h, off, count, seg);
-      if (count <= 0) continue;
-      const int s = (int)(j % stages);
-      const unsigned k = (unsigned)(j / stages);
-      if (seg != cur_seg) {
-        cur_seg = seg;
-        if (lane < p.n) sc0 = p.scales[(long long)lane * p.S + seg];
-        if (lane + 32 < p.n) sc1 = p.scales[(long long)(lane + 32) * p.S + seg];
+    int s = 0;
+    unsigned ph = 0;
+    int issued = 0;
+    Tile t = my_tiles > 0 ? ptiles[blockIdx.x] : Tile{0, 0, 0};
+    for (int j = 0; j < my_tiles; ++j) {
+      // next tile's descriptor is fetched while this one is issued
+      Tile tn = t;
+      if (j + 1 < my_tiles) tn = ptiles[blockIdx.x + (long long)(j + 1) * gridDim.x];
+      if (t.seg != cur_seg) {
+        cur_seg = t.seg;
+        if (lane < n) sc0 = p.scales[(long long)lane * p.S + t.seg];
+        if (lane + 32 < n) sc1 = p.scales[(long long)(lane + 32) * p.S + t.seg];
       }
-      if (k > 0) {
-        bool ok = true;
-        if (lane == 0) ok = mbar_wait_bounded(&ps->empty[s], (k - 1) & 1, abort_flag, p.status);
-        ok = __shfl_sync(0xffffffffu, ok, 0);
-        if (!ok) break;
-      } else if (*abort_flag) {
-        break;
+      // a fresh barrier passes a wait on the parity opposite to its first phase
+      bool ok = true;
+      if (lane == 0) ok = mbar_wait_bounded(&ps->empty[s], ph ^ 1u, abort_flag, p.status);
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      unsigned char* st = stage_base + (size_t)s * stage_bytes;
+      float2* s_scale = reinterpret_cast<float2*>(st + scales_off);
+      if (lane < n) s_scale[lane] = make_float2(sc0, sc0);
+      if (lane + 32 < n) s_scale[lane + 32] = make_float2(sc1, sc1);
+      if (lane == 0) {
+        StageHeader* hd = reinterpret_cast<StageHeader*>(st);
+        hd->off = t.off;
+        hd->count = t.count;
       }
-      unsigned char* st = stage_ptr(s);
-      float* s_scale = reinterpret_cast<float*>(st + (size_t)kState * kPipeTile * 4 + (size_t)p.n * (kPipeTile / 4));
-      if (lane < p.n) s_scale[lane] = sc0;
-      if (lane + 32 < p.n) s_scale[lane + 32] = sc1;
       __syncwarp();
-      const unsigned fbytes = (unsigned)count * 4u;
-      const unsigned cbytes = (unsigned)count / 4u;
-      if (lane == 0) mbar_arrive_expect_tx(&ps->full[s], kState * fbytes + (unsigned)p.n * cbytes);
+      const unsigned fbytes = (unsigned)t.count * 4u;
+      const unsigned cbytes = (unsigned)t.count / 4u;
+      if (lane == 0) mbar_arrive_expect_tx(&ps->full[s], kState * fbytes + (unsigned)n * cbytes);
       __syncwarp();
-      if (lane == 0) bulk_load(st, p.x + off, fbytes, &ps->full[s]);
+      float* sx = reinterpret_cast<float*>(st + kStageHeaderBytes);
+      if (lane == 0) bulk_load(sx, p.x + t.off, fbytes, &ps->full[s]);
       if (SERVER_MOMENTS) {
-        if (lane == 1) bulk_load(st + kPipeTile * 4, p.m + off, fbytes, &ps->full[s]);
-        if (lane == 2) bulk_load(st + 2 * kPipeTile * 4, p.v + off, fbytes, &ps->full[s]);
+        if (lane == 1) bulk_load(sx + kPipeTile, p.m + t.off, fbytes, &ps->full[s]);
+        if (lane == 2) bulk_load(sx + 2 * kPipeTile, p.v + t.off, fbytes, &ps->full[s]);
       }
-      unsigned char* s_codes = st + (size_t)kState * kPipeTile * 4;
-      for (int i = lane; i < p.n; i += 32) {
-        bulk_load(s_codes + (size_t)i * (kPipeTile / 4), p.gcodes + (long long)i * p.gcode_bytes + (off >> 2),
+      unsigned char* s_codes = st + kCodesOff;
+      for (int i = lane; i < n; i += 32) {
+        bulk_load(s_codes + (size_t)i * (kPipeTile / 4), p.gcodes + (long long)i * p.gcode_bytes + (t.off >> 2),
                   cbytes, &ps->full[s]);
       }
-      ++j;
+      ++issued;
+      if (++s == stages) { s = 0; ph ^= 1u; }
+      t = tn;
     }
-    // drain: nothing may still be landing in shared memory when the CTA exits
+    // drain after an abort: nothing may still be landing in shared memory when the CTA exits
     __syncwarp();
     if (lane == 0 && *abort_flag) {
-      for (long long jj = (j > stages ? j - stages : 0); jj < j; ++jj) {
-        const int s = (int)(jj % stages);
-        const unsigned k = (unsigned)(jj / stages);
+      const int back = issued < stages ? issued : stages;
+      int ds = s;
+      unsigned dph = ph;
+      for (int b = 0; b < back; ++b) {
+        if (--ds < 0) { ds = stages - 1; dph ^= 1u; }
         for (unsigned it = 0; it < kSpinLimit; ++it) {
-          if (mbar_try_wait(&ps->full[s], k & 1)) break;
+          if (mbar_try_wait(&ps->full[ds], dph)) break;
           __nanosleep(100);
         }
       }
     }
   } else if (warp == kPipeConsumers / 32 + 1) {
     // ------------------------------------------------------------------ storer
-    long long j = 0;
-    for (long long h = blockIdx.x; h < num_halves; h += gridDim.x) {
-      long long off; int count, seg;
-      half_tile(h, off, count, seg);
-      if (count <= 0) continue;
-      const int s = (int)(j % stages);
-      const unsigned k = (unsigned)(j / stages);
+    int s = 0;
+    unsigned ph = 0;
+    for (int j = 0; j < my_tiles; ++j) {
       bool ok = true;
-      if (lane == 0) ok = mbar_wait_bounded(&ps->computed[s], k & 1, abort_flag, p.status);
+      if (lane == 0) ok = mbar_wait_bounded(&ps->computed[s], ph, abort_flag, p.status);
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       if (lane == 0) {
-        unsigned char* st = stage_ptr(s);
-        const unsigned fbytes = (unsigned)count * 4u;
-        bulk_store(p.x + off, st, fbytes);
+        unsigned char* st = stage_base + (size_t)s * stage_bytes;
+        const StageHeader hd = *reinterpret_cast<const StageHeader*>(st);
+        float* sx = reinterpret_cast<float*>(st + kStageHeaderBytes);
+        const unsigned fbytes = (unsigned)hd.count * 4u;
+        bulk_store(p.x + hd.off, sx, fbytes);
         if (SERVER_MOMENTS) {
-          bulk_store(p.m + off, st + kPipeTile * 4, fbytes);
-          bulk_store(p.v + off, st + 2 * kPipeTile * 4, fbytes);
+          bulk_store(p.m + hd.off, sx + kPipeTile, fbytes);
+          bulk_store(p.v + hd.off, sx + 2 * kPipeTile, fbytes);
         }
         bulk_commit();
         bulk_wait_read_all();                    // the stage has been read out
         mbar_arrive(&ps->empty[s]);
       }
-      ++j;
+      if (++s == stages) { s = 0; ph ^= 1u; }
     }
     if (lane == 0) bulk_wait_all();               // writes are complete before the kernel ends
   } else {
     // ------------------------------------------------------------------ consumers
-    long long j = 0;
-    for (long long h = blockIdx.x; h < num_halves; h += gridDim.x) {
-      long long off; int count, seg;
-      half_tile(h, off, count, seg);
-      if (count <= 0) continue;
-      const int s = (int)(j % stages);
-      const unsigned k = (unsigned)(j / stages);
-      // every lane waits for itself; the warp then agrees on the outcome so that it never splits
-      if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->full[s], k & 1, abort_flag, p.status))) break;
-      unsigned char* st = stage_ptr(s);
-      const bool act = tid * 4 < count;                 // warp-uniform
-      if (act) {
-        float* sx = reinterpret_cast<float*>(st) + tid * 4;
-        const unsigned char* s_codes = st + (size_t)kState * kPipeTile * 4 + tid;
-        const float* s_scale = reinterpret_cast<const float*>(st + (size_t)kState * kPipeTile * 4 +
-                                                               (size_t)p.n * (kPipeTile / 4));
-        float acc[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+    // Two groups of 8 warps take alternate tiles, so that one group computes while
+    // the other waits for its data or hands its tile to the storer.  In a tile a
+    // thread owns elements 4t..4t+3 of both 1024-element rows.
+    const int group = tid / kPipeGroupThreads;
+    const int gt = tid - group * kPipeGroupThreads;           // 0..255
+    const int gwarp = gt >> 5;
+    int s = 0;
+    unsigned ph = 0;
+    // -(2^E + 1) for the four code positions of a byte (E = 23, 21, 19, 17)
+    const float2 k01 = make_float2(-(exp2i(23) + 1.0f), -(exp2i(21) + 1.0f));
+    const float2 k23 = make_float2(-(exp2i(19) + 1.0f), -(exp2i(17) + 1.0f));
+    const unsigned mg[4] = {opaque_u32(150u << 23), opaque_u32(148u << 23), opaque_u32(146u << 23),
+                            opaque_u32(144u << 23)};
+    for (int j = 0; j < my_tiles; ++j) {
+      if ((j & 1) == group) {
+        // every lane waits for itself; the warp then agrees on the outcome so that it never splits
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->full[s], ph, abort_flag, p.status))) break;
+        unsigned char* st = stage_base + (size_t)s * stage_bytes;
+        const StageHeader hd = *reinterpret_cast<const StageHeader*>(st);
+        const bool act0 = gt * 4 < hd.count;                   // warp-uniform
+        const bool act1 = kPipeTile / 2 + gt * 4 < hd.count;
+        if (act0) {
+          float* sx = reinterpret_cast<float*>(st + kStageHeaderBytes) + gt * 4;
+          const unsigned char* s_codes = st + kCodesOff + gt;
+          const float2* s_scale = reinterpret_cast<const float2*>(st + scales_off);
+          float2 a[4];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) a[c] = make_float2(0.0f, 0.0f);
+          if constexpr (NW > 0) {
+#pragma unroll
+            for (int i = 0; i < NW; ++i) {
+              decode_accumulate(s_scale[i], s_codes[i * (kPipeTile / 4)],
+                                s_codes[i * (kPipeTile / 4) + kPipeTile / 8], k01, k23, mg, a);
+            }
+          } else {
 #pragma unroll 4
-        for (int i = 0; i < p.n; ++i) {
-          const float sc = s_scale[i];
-          const unsigned b = s_codes[(size_t)i * (kPipeTile / 4)];
+            for (int i = 0; i < n; ++i) {
+              decode_accumulate(s_scale[i], s_codes[i * (kPipeTile / 4)],
+                                s_codes[i * (kPipeTile / 4) + kPipeTile / 8], k01, k23, mg, a);
+            }
+          }
+          // pads beyond the tile's length decode whatever the stage held; they are not used
+          float2 d[4];
+          if (inv_n_exact) {
+            const float2 inv = make_float2(p.inv_nf, p.inv_nf);
 #pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            const unsigned bits = (b & (3u << (2 * c))) | ((unsigned)(150 - 2 * c) << 23);
-            const float q = __fadd_rn(__uint_as_float(bits), -(exp2i(23 - 2 * c) + 1.0f));
-            acc[c] = __fmaf_rn(q, sc, acc[c]);
+            for (int c = 0; c < 4; ++c) d[c] = mul2_rn(a[c], inv);
+          } else {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) d[c] = make_float2(__fdiv_rn(a[c].x, p.nf), __fdiv_rn(a[c].y, p.nf));
+          }
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            if (r == 1 && !act1) break;
+            float* rx = sx + r * (kPipeTile / 2);
+            const float4 x4 = *reinterpret_cast<const float4*>(rx);
+            float xx[4];
+            if constexpr (SERVER_MOMENTS) {
+              float* rm = rx + kPipeTile;
+              float* rv = rx + 2 * kPipeTile;
+              const float4 m4 = *reinterpret_cast<const float4*>(rm);
+              const float4 v4 = *reinterpret_cast<const float4*>(rv);
+              float2 m01 = make_float2(m4.x, m4.y), m23 = make_float2(m4.z, m4.w);
+              float2 v01 = make_float2(v4.x, v4.y), v23 = make_float2(v4.z, v4.w);
+              moments2(p.h, d[2 * r], m01, v01);
+              moments2(p.h, d[2 * r + 1], m23, v23);
+              xx[0] = __fsub_rn(x4.x, adam_step(p.h, m01.x, v01.x, p.alpha));
+              xx[1] = __fsub_rn(x4.y, adam_step(p.h, m01.y, v01.y, p.alpha));
+              xx[2] = __fsub_rn(x4.z, adam_step(p.h, m23.x, v23.x, p.alpha));
+              xx[3] = __fsub_rn(x4.w, adam_step(p.h, m23.y, v23.y, p.alpha));
+              *reinterpret_cast<float4*>(rm) = make_float4(m01.x, m01.y, m23.x, m23.y);
+              *reinterpret_cast<float4*>(rv) = make_float4(v01.x, v01.y, v23.x, v23.y);
+            } else {
+              xx[0] = __fsub_rn(x4.x, d[2 * r].x);
+              xx[1] = __fsub_rn(x4.y, d[2 * r].y);
+              xx[2] = __fsub_rn(x4.z, d[2 * r + 1].x);
+              xx[3] = __fsub_rn(x4.w, d[2 * r + 1].y);
+            }
+            *reinterpret_cast<float4*>(rx) = make_float4(xx[0], xx[1], xx[2], xx[3]);
+            if (p.kx >= 0) {
+              const long long e0 = hd.off + r * (kPipeTile / 2);
+              broadcast_row(xx, p.kx, p.xbits, p.wcodes, p.wresid, e0 + gt * 4, e0 + gwarp * 128, lane);
+            }
           }
         }
-        const float4 x4 = *reinterpret_cast<const float4*>(sx);
-        float xx[4] = {x4.x, x4.y, x4.z, x4.w};
-        float dh[4];
-#pragma unroll
-        for (int c = 0; c < 4; ++c)
-          dh[c] = inv_n_exact ? __fmul_rn(acc[c], p.inv_nf) : __fdiv_rn(acc[c], p.nf);
-        if constexpr (SERVER_MOMENTS) {
-          float* sm = sx + kPipeTile;
-          float* sv = sx + 2 * kPipeTile;
-          const float4 m4 = *reinterpret_cast<const float4*>(sm);
-          const float4 v4 = *reinterpret_cast<const float4*>(sv);
-          float mm[4] = {m4.x, m4.y, m4.z, m4.w};
-          float vs[4] = {v4.x, v4.y, v4.z, v4.w};
-#pragma unroll
-          for (int c = 0; c < 4; ++c) {
-            moments(p.h, dh[c], mm[c], vs[c]);
-            xx[c] = __fsub_rn(xx[c], adam_step(p.h, mm[c], vs[c], p.alpha));
-          }
-          *reinterpret_cast<float4*>(sm) = make_float4(mm[0], mm[1], mm[2], mm[3]);
-          *reinterpret_cast<float4*>(sv) = make_float4(vs[0], vs[1], vs[2], vs[3]);
-        } else {
-#pragma unroll
-          for (int c = 0; c < 4; ++c) xx[c] = __fsub_rn(xx[c], dh[c]);
-        }
-        *reinterpret_cast<float4*>(sx) = make_float4(xx[0], xx[1], xx[2], xx[3]);
-        if (p.kx >= 0) {
-          broadcast_row(xx, p.kx, p.xbits, p.wcodes, p.wresid, off + tid * 4, off + warp * 128, lane);
-        }
+        fence_async_shared();                              // my writes, before the storer's bulk reads
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ps->computed[s]);
       }
-      fence_async_shared();                              // my writes, before the storer's bulk reads
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&ps->computed[s]);
-      ++j;
+      if (++s == stages) { s = 0; ph ^= 1u; }
     }
   }
   __syncthreads();
