@@ -146,6 +146,7 @@ struct qadam_ctx {
   // persistent pipelined server pass (ternary codes): stages > 0 when in use
   int pipe_stages = 0;
   size_t pipe_smem = 0;
+  CUtensorMap codes_map;
   // instrumentation: event pairs of the launches since the last read
   bool profiling = false;
   struct Timed { int kind; cudaEvent_t start, stop; };
@@ -197,7 +198,7 @@ ServerKernel pick_server(const qadam_ctx* c) {
   }
 }
 
-using PipeKernel = void (*)(const ServerParams, const Tile*, int, int, int);
+using PipeKernel = void (*)(const ServerParams, const CUtensorMap, const Tile*, int, int, int);
 
 template <bool SM>
 PipeKernel pick_pipe_n(int n) {
@@ -357,7 +358,8 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
     const bool want_plain = env && std::strcmp(env, "plain") == 0;
     int stages = (int)(((size_t)max_smem - 256) / sb);
     stages = std::min(stages, kPipeMaxStages);
-    if (!want_plain && c->geo.gmode == G_TERNARY && cfg->n <= kPipeMaxWorkers && stages >= 2) {
+    if (!want_plain && c->geo.gmode == G_TERNARY && cfg->n <= kPipeMaxWorkers && stages >= 2 &&
+        make_codes_tensor_map(&c->codes_map, b->gcodes, (long long)c->geo.gcode_bytes, cfg->n)) {
       c->pipe_stages = stages;
       c->pipe_smem = 256 + (size_t)stages * sb;
       if (!cuda_ok(cudaFuncSetAttribute(pick_pipe(c), cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -470,7 +472,8 @@ int qadam_server_step(qadam_ctx* c, int64_t step, float lr_t) {
       const int inv_exact = (n & (n - 1)) == 0 ? 1 : 0;
       const int np = (int)c->geo.ptiles.size();
       const int pgrid = std::min(c->sm_count, np);
-      pick_pipe(c)<<<pgrid, kPipeThreads, c->pipe_smem, c->stream>>>(p, c->d_ptiles, np, c->pipe_stages, inv_exact);
+      pick_pipe(c)<<<pgrid, kPipeThreads, c->pipe_smem, c->stream>>>(p, c->codes_map, c->d_ptiles, np,
+                                                                      c->pipe_stages, inv_exact);
     } else {
       pick_server(c)<<<grid, kThreads, c->server_smem, c->stream>>>(p);
     }

@@ -14,6 +14,8 @@
 // its loop, outstanding copies are drained and the kernel returns.
 #pragma once
 
+#include <cuda.h>
+
 #include "qadam_kernels.cuh"
 
 namespace qadam {
@@ -59,6 +61,16 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, unsi
       "l"(gsrc), "r"(bytes), "r"(smem_u32(bar))
       : "memory");
 }
+// One tiled 2-D tensor copy global -> shared: the box of `map` whose corner is at
+// (c0, c1) in elements; completion counted in bytes (always the whole box) on `bar`.
+__device__ __forceinline__ void tensor_load_2d(void* smem_dst, const CUtensorMap* map, int c0, int c1,
+                                               unsigned long long* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(smem_dst)),
+      "l"(map), "r"(c0), "r"(c1), "r"(smem_u32(bar))
+      : "memory");
+}
 // shared -> global, tracked by the issuing thread's bulk async-group
 __device__ __forceinline__ void bulk_store(void* gdst, const void* smem_src, unsigned bytes) {
   asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst),
@@ -88,6 +100,32 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsig
   *abort_flag = 1;
   atomicOr(status, 2u);
   return false;
+}
+
+// Tensor map over the n packed 2-bit code streams, seen as a 2-D array of 32-bit
+// words [n rows][gcode_bytes / 4], with a box of one tile's words (kPipeTile / 16)
+// by all n rows: one request brings every worker's codes of a tile, row after row,
+// into shared memory.  Encoded through the driver entry point the runtime hands out,
+// so the library links against the runtime only.  Returns false if unavailable.
+inline bool make_codes_tensor_map(CUtensorMap* map, const void* gcodes, long long gcode_bytes, int n) {
+  typedef CUresult (*EncodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
+                                  CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                  CUtensorMapFloatOOBfill);
+  void* fn = nullptr;
+  cudaDriverEntryPointQueryResult qres;
+  if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
+      qres != cudaDriverEntryPointSuccess || fn == nullptr)
+    return false;
+  const cuuint64_t dims[2] = {(cuuint64_t)(gcode_bytes / 4), (cuuint64_t)n};
+  const cuuint64_t strides[1] = {(cuuint64_t)gcode_bytes};          // bytes between rows
+  const cuuint32_t box[2] = {(cuuint32_t)(kPipeTile / 16), (cuuint32_t)n};
+  const cuuint32_t estr[2] = {1, 1};
+  const CUresult r = reinterpret_cast<EncodeTiled>(fn)(
+      map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(gcodes), dims, strides, box, estr,
+      CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+      CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
 }
 
 struct PipeSmem {
@@ -171,8 +209,9 @@ __device__ __forceinline__ unsigned opaque_u32(unsigned v) {
 // every shared-memory offset is an immediate).  NW = 0: p.n workers, run-time loop.
 template <bool SERVER_MOMENTS, int NW>
 __global__ void __launch_bounds__(kPipeThreads, 1)
-server_pipe_kernel(const ServerParams p, const Tile* __restrict__ ptiles, const int num_ptiles,
-                   const int stages, const int inv_n_exact) {
+server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap codes_map,
+                   const Tile* __restrict__ ptiles, const int num_ptiles, const int stages,
+                   const int inv_n_exact) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   PipeSmem* ps = reinterpret_cast<PipeSmem*>(smem_raw);
   unsigned char* stage_base = smem_raw + 256;
@@ -232,20 +271,19 @@ server_pipe_kernel(const ServerParams p, const Tile* __restrict__ ptiles, const 
         hd->count = t.count;
       }
       __syncwarp();
-      const unsigned fbytes = (unsigned)t.count * 4u;
-      const unsigned cbytes = (unsigned)t.count / 4u;
-      if (lane == 0) mbar_arrive_expect_tx(&ps->full[s], kState * fbytes + (unsigned)n * cbytes);
-      __syncwarp();
-      float* sx = reinterpret_cast<float*>(st + kStageHeaderBytes);
-      if (lane == 0) bulk_load(sx, p.x + t.off, fbytes, &ps->full[s]);
-      if (SERVER_MOMENTS) {
-        if (lane == 1) bulk_load(sx + kPipeTile, p.m + t.off, fbytes, &ps->full[s]);
-        if (lane == 2) bulk_load(sx + 2 * kPipeTile, p.v + t.off, fbytes, &ps->full[s]);
-      }
-      unsigned char* s_codes = st + kCodesOff;
-      for (int i = lane; i < n; i += 32) {
-        bulk_load(s_codes + (size_t)i * (kPipeTile / 4), p.gcodes + (long long)i * p.gcode_bytes + (t.off >> 2),
-                  cbytes, &ps->full[s]);
+      // one elected lane issues the tile's four requests: x, m, v runs and the code box.
+      // The box always carries n full 512-byte rows (beyond a short tile's length it holds
+      // the neighbouring codes or zero fill, which nobody reads).
+      if (lane == 0) {
+        const unsigned fbytes = (unsigned)t.count * 4u;
+        mbar_arrive_expect_tx(&ps->full[s], kState * fbytes + (unsigned)n * (kPipeTile / 4));
+        float* sx = reinterpret_cast<float*>(st + kStageHeaderBytes);
+        bulk_load(sx, p.x + t.off, fbytes, &ps->full[s]);
+        if (SERVER_MOMENTS) {
+          bulk_load(sx + kPipeTile, p.m + t.off, fbytes, &ps->full[s]);
+          bulk_load(sx + 2 * kPipeTile, p.v + t.off, fbytes, &ps->full[s]);
+        }
+        tensor_load_2d(st + kCodesOff, &codes_map, (int)(t.off >> 4), 0, &ps->full[s]);
       }
       ++issued;
       if (++s == stages) { s = 0; ph ^= 1u; }
