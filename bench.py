@@ -41,6 +41,10 @@ FALLBACK_HBM_GBS = 6650.0
 # whose digest is recorded beside it.
 NCU_TRAFFIC = {
     # kernel: (bytes per unit, digest of csrc/ at capture time)
+    # profiles/step_kernels_flat25_n16_server_moments.md (flat25, n = 16, moments on the server)
+    "absmax": (8.012, "9f6de76b895cb432"),
+    "quantize": (12.150, "9f6de76b895cb432"),
+    "server": (26.52, "9f6de76b895cb432"),
 }
 
 
@@ -197,7 +201,7 @@ def time_oracle(w, placement: str, sample_log2: int, steps: int, warmup: int):
 
 
 def run_reference(args):
-    rank = int(os.environ.get("RANK", "0"))
+    rank, _, _ = rank_env()
     if rank != 0:
         return
     w = get_workload(args)
@@ -231,6 +235,30 @@ def workload_config(w, args, extra=None):
     return cfg
 
 
+# ----------------------------------------------------------------------------- ranks
+
+def rank_env():
+    """(rank, world size, local rank) as torch.distributed.run exports them."""
+    return (int(os.environ.get("RANK", "0")), int(os.environ.get("WORLD_SIZE", "1")),
+            int(os.environ.get("LOCAL_RANK", "0")))
+
+
+def max_over_ranks(ms: float, world: int, device) -> float:
+    """The slowest rank's time: replicas finish when the last one does."""
+    if world <= 1:
+        return float(ms)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def job_value(d: int, n_workers: int, world: int, ms_per_step: float) -> float:
+    """Whole-job elements per second: every rank steps its own replica of d*n elements."""
+    return world * d * n_workers / (ms_per_step * 1e-3)
+
+
 # ----------------------------------------------------------------------------- the CUDA path
 
 def run_b200(args):
@@ -239,9 +267,7 @@ def run_b200(args):
     import qadam_inputs as qi
     import paper_2004_14180_b200 as qb
 
-    rank = int(os.environ.get("RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = rank_env()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU path); "
                          "use --impl reference for the oracle")
@@ -299,12 +325,9 @@ def run_b200(args):
     gpu_launches = q.launches - launches0
     status = q.poll_status()
 
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_total = float(t.item())
+    ms_total = max_over_ranks(ms_total, world, dev)
     ms_step = ms_total / args.steps
-    value = world * w.d * w.n / (ms_step * 1e-3)
+    value = job_value(w.d, w.n, world, ms_step)
 
     # ---- end to end through the host-buffer entry point -------------------------------
     e2e = None
@@ -323,11 +346,8 @@ def run_b200(args):
             q.step_host(step, g_host, g, out_host)
         s1.record()
         sync_all()
-        te = torch.tensor([s0.elapsed_time(s1)], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(te, op=dist.ReduceOp.MAX)
-        ms_e2e = float(te.item()) / args.e2e_steps
-        e2e = {"value": world * w.d * w.n / (ms_e2e * 1e-3), "unit": UNIT,
+        ms_e2e = max_over_ranks(s0.elapsed_time(s1), world, dev) / args.e2e_steps
+        e2e = {"value": job_value(w.d, w.n, world, ms_e2e), "unit": UNIT,
                "h2d_bytes_per_step": w.n * D * 4, "d2h_bytes_per_step": out_bytes,
                "steps": args.e2e_steps, "ms_per_step": ms_e2e,
                "api": "qadam_step_host (pinned host gradients in, packed broadcast out)"}
