@@ -77,7 +77,8 @@ enum qadam_error {
   QADAM_ERR_WORKER = -7,      /* worker range outside 0..n                          */
   QADAM_ERR_HYPER = -8,       /* beta/theta outside [0,1), eps <= 0 or a bad step size */
   QADAM_ERR_CUDA = -9,        /* a CUDA call failed; see qadam_last_cuda_error      */
-  QADAM_ERR_PLACEMENT = -10   /* placement is not one of the two values             */
+  QADAM_ERR_PLACEMENT = -10,  /* placement is not one of the two values             */
+  QADAM_ERR_CAPACITY = -11    /* beyond the fixed capacity of qadam_worker_scales_static */
 };
 
 /* Bits of the device status word. */
@@ -169,6 +170,29 @@ int qadam_server_step(qadam_ctx* ctx, int64_t step, float lr_t);
  * stream before returning.  out_host may be NULL to skip the read-back. */
 int qadam_step_host(qadam_ctx* ctx, int64_t step, const float* g_host, float* g_stage,
                     void* out_host, float lr_t);
+
+/* Worker scales without any allocation (no counterpart in the paper: a service
+ * entry point for callers that cannot allocate device memory at all, such as a
+ * process that sizes its device memory once at start-up and forbids cudaMalloc
+ * afterwards, and therefore cannot provide the workspace the context-based calls
+ * need).
+ *   scales[i] = max_j |g[i][j] + e[i][j]|,  i = 0..n-1,
+ * i.e. exactly what qadam_worker_compress writes into `scales` for a problem with
+ * num_segments = 1 and the moments on the server (bit-identical).  g, e: device,
+ * [n][D] binary32, 16-byte aligned, D a multiple of 128 (pads zero); scales: device,
+ * [n] out; stream: cudaStream_t.  Enqueues on `stream` and returns.
+ * The kernel's scratch (tile table, running maxima) is a fixed 260 KiB array inside
+ * the library image, held by every GPU that loads the library until the process
+ * ends.  Limits: D <= QADAM_STATIC_MAX_ELEMENTS and n <= QADAM_STATIC_MAX_WORKERS,
+ * else QADAM_ERR_CAPACITY and nothing is enqueued.  The call allocates and frees
+ * nothing.  The first call on each device looks the array's address up; make that
+ * first call outside any stream capture.  All calls on a device share the one
+ * array (each call rewrites and clears what it uses), so two calls that may overlap
+ * on the GPU (different streams, no dependency between them) race: serialise them. */
+#define QADAM_STATIC_MAX_ELEMENTS (1ll << 26)
+#define QADAM_STATIC_MAX_WORKERS 1024
+int qadam_worker_scales_static(const float* g, const float* e, int64_t D, int32_t n,
+                               float* scales, void* stream);
 
 /* Waits for the context's stream, then copies the status word to *host_status. */
 int qadam_poll_status(qadam_ctx* ctx, uint32_t* host_status);

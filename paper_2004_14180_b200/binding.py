@@ -23,8 +23,11 @@ exported_symbols = (
     "qadam_query_sizes", "qadam_grad_code_bits", "qadam_weight_code_bits", "qadam_create",
     "qadam_worker_compress", "qadam_server_step", "qadam_step_host", "qadam_poll_status",
     "qadam_launch_count", "qadam_destroy", "qadam_strerror", "qadam_last_cuda_error",
-    "qadam_profile_enable", "qadam_profile_read",
+    "qadam_profile_enable", "qadam_profile_read", "qadam_worker_scales_static",
 )
+
+STATIC_MAX_ELEMENTS = 1 << 26
+STATIC_MAX_WORKERS = 1024
 
 KERNEL_NAMES = ("absmax", "quantize", "identity", "server", "broadcast")
 
@@ -96,6 +99,8 @@ def load_library():
     L.qadam_profile_enable.argtypes = [C.c_void_p, C.c_int]
     L.qadam_profile_read.restype = C.c_int
     L.qadam_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    L.qadam_worker_scales_static.restype = C.c_int
+    L.qadam_worker_scales_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p]
     L.qadam_launch_count.restype = C.c_int64
     L.qadam_launch_count.argtypes = [C.c_void_p]
     L.qadam_destroy.restype = C.c_int
@@ -177,6 +182,14 @@ def qadam_profile_read(ctx: int):
     ms, cnt = (C.c_double * n)(), (C.c_int64 * n)()
     _check(load_library().qadam_profile_read(ctx, ms, cnt), "qadam_profile_read")
     return {KERNEL_NAMES[i]: (ms[i], cnt[i]) for i in range(n)}
+
+
+def qadam_worker_scales_static(g_ptr: int, e_ptr: int, D: int, n: int, scales_ptr: int,
+                               stream_ptr: Optional[int] = None) -> None:
+    """Max-abs scales of n workers without a context, a workspace or any allocation
+    (for callers that cannot allocate device memory); see include/qadam.h."""
+    _check(load_library().qadam_worker_scales_static(g_ptr, e_ptr, D, n, scales_ptr, stream_ptr),
+           "qadam_worker_scales_static")
 
 
 def qadam_launch_count(ctx: int) -> int:

@@ -565,6 +565,7 @@ const char* qadam_strerror(int err) {
     case QADAM_ERR_HYPER: return "invalid beta, theta, epsilon or step size";
     case QADAM_ERR_CUDA: return "a CUDA call failed";
     case QADAM_ERR_PLACEMENT: return "invalid placement";
+    case QADAM_ERR_CAPACITY: return "size beyond the fixed capacity of the allocation-free entry point";
     default: return "unknown error";
   }
 }

@@ -291,8 +291,9 @@ __device__ __forceinline__ void broadcast_row(const float xx[4], int kx, int xbi
   }
 }
 
-// Stand-alone Q_x(x) (the broadcast of x_1 before the first step).
-__global__ void __launch_bounds__(kThreads)
+// Stand-alone Q_x(x) (the broadcast of x_1 before the first step).  Internal linkage:
+// this header is included by more than one source file of the library.
+static __global__ void __launch_bounds__(kThreads)
 weight_broadcast_kernel(const ServerParams p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   for (int t = blockIdx.x; t < p.tiles_per_worker; t += gridDim.x) {
