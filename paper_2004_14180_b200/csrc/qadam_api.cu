@@ -357,7 +357,7 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
     const char* env = std::getenv("QADAM_SERVER_KERNEL");
     const bool want_plain = env && std::strcmp(env, "plain") == 0;
     int stages = (int)(((size_t)max_smem - 256) / sb);
-    stages = std::min(stages, kPipeMaxStages);
+    stages = pipe_legal_stages(std::min(stages, kPipeMaxStages));
     if (!want_plain && c->geo.gmode == G_TERNARY && cfg->n <= kPipeMaxWorkers && stages >= 2 &&
         make_codes_tensor_map(&c->codes_map, b->gcodes, (long long)c->geo.gcode_bytes, cfg->n)) {
       c->pipe_stages = stages;

@@ -21,8 +21,12 @@
 namespace qadam {
 
 constexpr int kPipeTile = 2048;                 // elements per pipeline tile
-constexpr int kPipeConsumers = 512;             // 16 warps, 4 elements per thread
-constexpr int kPipeGroupThreads = 256;          // two consumer groups take alternate tiles
+#ifndef QADAM_PIPE_GROUPS
+#define QADAM_PIPE_GROUPS 2
+#endif
+constexpr int kPipeGroups = QADAM_PIPE_GROUPS;  // consumer groups; group g takes tiles g, g + groups, ...
+constexpr int kPipeGroupThreads = 256;          // 8 warps per group, 8 elements per thread and tile
+constexpr int kPipeConsumers = kPipeGroups * kPipeGroupThreads;
 constexpr int kPipeThreads = kPipeConsumers + 64;   // + producer warp + storer warp
 constexpr int kPipeMaxWorkers = 64;
 constexpr int kPipeMaxStages = 8;
@@ -126,6 +130,16 @@ inline bool make_codes_tensor_map(CUtensorMap* map, const void* gcodes, long lon
       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
+}
+
+// The ring must hold a multiple of kPipeGroups stages.  A stage is then always served by
+// the same consumer group, so a thread that waits on a stage's barrier for use k + 1 has
+// itself seen use k complete.  With any other count the groups would alternate on a stage,
+// and a group running ahead could ask for the parity of use k + 1 while use k is still in
+// flight, which the barrier answers with "complete" (it reports the phase before the
+// current one): the group would then work on a stage that has not been loaded.
+__host__ __device__ inline int pipe_legal_stages(int stages) {
+  return stages / kPipeGroups * kPipeGroups;
 }
 
 struct PipeSmem {
@@ -344,8 +358,11 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
     const float2 k23 = make_float2(-(exp2i(19) + 1.0f), -(exp2i(17) + 1.0f));
     const unsigned mg[4] = {opaque_u32(150u << 23), opaque_u32(148u << 23), opaque_u32(146u << 23),
                             opaque_u32(144u << 23)};
+    bool sparse_mode = true;          // warp-uniform: look for workers with nothing but level 0
+    int dense_tiles_left = 0;
+    int dense_span = 8;
     for (int j = 0; j < my_tiles; ++j) {
-      if ((j & 1) == group) {
+      if (j % kPipeGroups == group) {
         // every lane waits for itself; the warp then agrees on the outcome so that it never splits
         if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->full[s], ph, abort_flag, p.status))) break;
         unsigned char* st = stage_base + (size_t)s * stage_bytes;
@@ -359,18 +376,55 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
           float2 a[4];
 #pragma unroll
           for (int c = 0; c < 4; ++c) a[c] = make_float2(0.0f, 0.0f);
-          if constexpr (NW > 0) {
+          // Zero skipping.  With a max-abs scale most ternary codes are level 0 (code 1,
+          // byte 0x55 for four of them), and a worker whose 256 codes in this warp's two
+          // rows are all level 0 adds +0 to every sum, which changes nothing (a sum is
+          // never -0).  The warp first votes, worker by worker and without branching, on
+          // whether any lane holds a code other than 1, then decodes only the workers that
+          // do, in increasing worker order (the order of the sum is unchanged).  When
+          // more than a third of the workers have something to add the warp stops
+          // looking for a while: dense codes would only pay for the votes.
+          auto contribute = [&](int i) {
+            decode_accumulate(s_scale[i], s_codes[i * (kPipeTile / 4)],
+                              s_codes[i * (kPipeTile / 4) + kPipeTile / 8], k01, k23, mg, a);
+          };
+          auto has_nonzero = [&](int i) -> unsigned long long {
+            const unsigned b0 = s_codes[i * (kPipeTile / 4)];
+            const unsigned b1 = s_codes[i * (kPipeTile / 4) + kPipeTile / 8];
+            return __any_sync(0xffffffffu, (b0 & b1 & 0x55u) != 0x55u) ? 1ull : 0ull;
+          };
+          if (sparse_mode) {
+            unsigned long long live = 0;
+            if constexpr (NW > 0) {
 #pragma unroll
-            for (int i = 0; i < NW; ++i) {
-              decode_accumulate(s_scale[i], s_codes[i * (kPipeTile / 4)],
-                                s_codes[i * (kPipeTile / 4) + kPipeTile / 8], k01, k23, mg, a);
+              for (int i = 0; i < NW; ++i) live |= has_nonzero(i) << i;
+            } else {
+#pragma unroll 4
+              for (int i = 0; i < n; ++i) live |= has_nonzero(i) << i;
+            }
+            if (3 * __popcll(live) > n) {
+              // too many live workers for the vote to pay: decode everything for a while,
+              // looking again after 16, 32, ... up to 1024 tiles
+              sparse_mode = false;
+              dense_span = dense_span < 1024 ? 2 * dense_span : 1024;
+              dense_tiles_left = dense_span;
+            } else {
+              dense_span = 8;
+            }
+            while (live) {
+              const int i = __ffsll((long long)live) - 1;
+              live &= live - 1;
+              contribute(i);
             }
           } else {
+            if constexpr (NW > 0) {
+#pragma unroll
+              for (int i = 0; i < NW; ++i) contribute(i);
+            } else {
 #pragma unroll 4
-            for (int i = 0; i < n; ++i) {
-              decode_accumulate(s_scale[i], s_codes[i * (kPipeTile / 4)],
-                                s_codes[i * (kPipeTile / 4) + kPipeTile / 8], k01, k23, mg, a);
+              for (int i = 0; i < n; ++i) contribute(i);
             }
+            if (--dense_tiles_left <= 0) sparse_mode = true;
           }
           // pads beyond the tile's length decode whatever the stage held; they are not used
           float2 d[4];

@@ -119,6 +119,29 @@ def test_heavy_tails_and_outliers():
     p.close()
 
 
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_sparse_and_dense_code_regions(placement):
+    """The server pass skips workers whose codes in a warp's rows are all level 0 and
+    falls back to decoding everything where codes are dense; a vector with a dense
+    third and a sparse rest, long enough that every CTA switches mode several times,
+    must still match the oracle bit for bit."""
+    rng = np.random.default_rng(77)
+    d, n = 1 << 25, 4
+    dense_end = d * 3 // 10
+    x1 = (rng.standard_normal(d) * 0.05).astype(np.float32)
+    p = Pair([d], n, 0, 0, placement, x1=x1)
+    for t in range(2):
+        g = (rng.standard_normal((n, d)) * 1e-4).astype(np.float32)
+        g[:, :dense_end] = rng.standard_normal((n, dense_end)).astype(np.float32)
+        hits = rng.integers(dense_end, d, (n, 400))
+        for i in range(n):
+            g[i, hits[i]] = np.where(rng.random(400) < 0.5, 4.0, -4.0)
+        g[:, d - 1] = 5.0
+        p.step(g, threads=4)
+    p.compare_state()
+    p.close()
+
+
 def test_nonfinite_input_sets_status_bit():
     import paper_2004_14180_b200 as qb
     q = qb.QAdam([1000], 1, kg=0, kx=-1)
