@@ -382,8 +382,9 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
           // never -0).  The warp first votes, worker by worker and without branching, on
           // whether any lane holds a code other than 1, then decodes only the workers that
           // do, in increasing worker order (the order of the sum is unchanged).  When
-          // more than a third of the workers have something to add the warp stops
-          // looking for a while: dense codes would only pay for the votes.
+          // more than an eighth of the workers have something to add the warp stops
+          // looking for a while: the votes cost about half a decode, so denser codes are
+          // decoded faster without them.
           auto contribute = [&](int i) {
             decode_accumulate(s_scale[i], s_codes[i * (kPipeTile / 4)],
                               s_codes[i * (kPipeTile / 4) + kPipeTile / 8], k01, k23, mg, a);
@@ -402,7 +403,7 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
 #pragma unroll 4
               for (int i = 0; i < n; ++i) live |= has_nonzero(i) << i;
             }
-            if (3 * __popcll(live) > n) {
+            if (8 * __popcll(live) > n) {
               // too many live workers for the vote to pay: decode everything for a while,
               // looking again after 16, 32, ... up to 1024 tiles
               sparse_mode = false;
