@@ -149,11 +149,21 @@ class ClockSampler:
 
 # ----------------------------------------------------------------------------- byte accounting
 
-def algorithmic_bytes(kernel: str, w, placement: str, D: int, gbits: int, xbits: int) -> float:
+def algorithmic_bytes(kernel: str, w, placement: str, D: int, gbits: int, xbits: int,
+                      pass_model=None) -> float:
     """Bytes one launch of `kernel` must move at its interface (fp32 state it has
-    to read and write, packed codes), for all n workers."""
+    to read and write, packed codes), for all n workers.  For the fused worker kernel
+    the figure is capacity aware: (worker, segment) pairs that fit the kernel's L2
+    group budget are counted once (one pass), larger ones twice (the max-abs scale
+    needs the whole pair before any of it can be quantized)."""
     n = w.n
     server_moments = placement == "server"
+    if kernel == "worker_fused":
+        one_pass, two_pass = pass_model
+        if server_moments:      # read g, e (twice when two-pass); write e and the codes
+            return one_pass * (12.0 + gbits / 8.0) + two_pass * (20.0 + gbits / 8.0)
+        # read g, m, v, e; write m, v, e and codes; two-pass adds a write and a read of u
+        return one_pass * (28.0 + gbits / 8.0) + two_pass * (36.0 + gbits / 8.0)
     if kernel == "absmax":      # phase 1: read g, e (worker moments: + read m, v, write m, v, u)
         per = 8.0 if server_moments else 28.0
         return per * n * D
@@ -360,7 +370,8 @@ def run_b200(args):
         if cnt == 0:
             continue
         per = ms / cnt
-        bytes_ = algorithmic_bytes(name, w, args.placement, D, q.gcode_bytes * 8 // D, q.wcode_bytes * 8 // D)
+        bytes_ = algorithmic_bytes(name, w, args.placement, D, q.gcode_bytes * 8 // D, q.wcode_bytes * 8 // D,
+                                   pass_model=q.worker_pass_model())
         kernels[name] = {"launches": int(cnt), "ms_per_launch": per,
                          "share": ms / sum(m for m, c in prof.values()),
                          "algorithmic_bytes": bytes_, "achieved_gbs": bytes_ / (per * 1e-3) / 1e9,
@@ -368,7 +379,7 @@ def run_b200(args):
     dom = max(kernels, key=lambda k: kernels[k]["launches"] * kernels[k]["ms_per_launch"])
     traffic = None
     if dom in NCU_TRAFFIC and NCU_TRAFFIC[dom][1] == csrc_digest():
-        units = w.n * D if dom in ("absmax", "quantize", "identity") else D
+        units = w.n * D if dom in ("absmax", "quantize", "identity", "worker_fused") else D
         traffic = NCU_TRAFFIC[dom][0] * units
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["achieved_gbs"],
                 "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",

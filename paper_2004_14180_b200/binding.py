@@ -24,12 +24,13 @@ exported_symbols = (
     "qadam_worker_compress", "qadam_server_step", "qadam_step_host", "qadam_poll_status",
     "qadam_launch_count", "qadam_destroy", "qadam_strerror", "qadam_last_cuda_error",
     "qadam_profile_enable", "qadam_profile_read", "qadam_worker_scales_static",
+    "qadam_worker_pass_model",
 )
 
 STATIC_MAX_ELEMENTS = 1 << 26
 STATIC_MAX_WORKERS = 1024
 
-KERNEL_NAMES = ("absmax", "quantize", "identity", "server", "broadcast")
+KERNEL_NAMES = ("absmax", "quantize", "identity", "server", "broadcast", "worker_fused")
 
 
 class QAdamError(RuntimeError):
@@ -101,6 +102,8 @@ def load_library():
     L.qadam_profile_read.argtypes = [C.c_void_p, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
     L.qadam_worker_scales_static.restype = C.c_int
     L.qadam_worker_scales_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p]
+    L.qadam_worker_pass_model.restype = C.c_int
+    L.qadam_worker_pass_model.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
     L.qadam_launch_count.restype = C.c_int64
     L.qadam_launch_count.argtypes = [C.c_void_p]
     L.qadam_destroy.restype = C.c_int
@@ -190,6 +193,13 @@ def qadam_worker_scales_static(g_ptr: int, e_ptr: int, D: int, n: int, scales_pt
     (for callers that cannot allocate device memory); see include/qadam.h."""
     _check(load_library().qadam_worker_scales_static(g_ptr, e_ptr, D, n, scales_ptr, stream_ptr),
            "qadam_worker_scales_static")
+
+
+def qadam_worker_pass_model(ctx: int):
+    """-> (one_pass, two_pass): (worker, element) pairs read from HBM once / twice by the worker side."""
+    a, b = C.c_int64(), C.c_int64()
+    _check(load_library().qadam_worker_pass_model(ctx, C.byref(a), C.byref(b)), "qadam_worker_pass_model")
+    return a.value, b.value
 
 
 def qadam_launch_count(ctx: int) -> int:
@@ -308,6 +318,9 @@ class QAdam:
 
     def profile_read(self):
         return qadam_profile_read(self.ctx)
+
+    def worker_pass_model(self):
+        return qadam_worker_pass_model(self.ctx)
 
     def poll_status(self) -> int:
         return qadam_poll_status(self.ctx)

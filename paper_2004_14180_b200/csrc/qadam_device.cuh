@@ -112,6 +112,27 @@ __device__ __forceinline__ float level_value(int c, int k) {
 // s = |u|_inf, returns the code (level index + L) and writes e' = u - Q_g(u).
 template <int MODE>
 __device__ __forceinline__ unsigned quantize_grad(float u, float s, int k, int L, float& e_next) {
+  if constexpr (MODE == G_TERNARY) {
+    // The decision is y = fl(|u| / s) > 1/2.  It is settled without dividing for all but
+    // a sliver of values: |u| <= s/2 gives a quotient <= 1/2 (s/2 is exact for a normal
+    // s), and |u| > (s/2)(1 + 2^-21) gives a quotient whose rounding stays above 1/2.
+    // Only values inside that band, and tiny or non-finite scales, take the division.
+    const float a = fabsf(u);
+    const float h = __fmul_rn(0.5f, s);
+    const float hi = __fmul_rn(h, 1.000000476837158203125f);       // 1 + 2^-21
+    bool one;
+    if (a <= h && s >= 1e-30f) {
+      one = false;
+    } else if (a > hi && s >= 1e-30f && s < 3.0e38f) {
+      one = true;
+    } else {
+      one = __fdiv_rn(a, s) > 0.5f;
+    }
+    const bool neg = u < 0.0f;
+    const float deq = one ? (neg ? -s : s) : 0.0f;
+    e_next = __fsub_rn(u, deq);
+    return one ? (neg ? 0u : 2u) : 1u;
+  }
   const float y = __fdiv_rn(fabsf(u), s);
   const int c = level_index<MODE>(y, k, L);
   const bool neg = u < 0.0f;
