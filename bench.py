@@ -41,10 +41,10 @@ FALLBACK_HBM_GBS = 6650.0
 # whose digest is recorded beside it.
 NCU_TRAFFIC = {
     # kernel: (bytes per unit, digest of csrc/ at capture time)
-    # profiles/step_kernels_flat25_n16_server_moments.md (flat25, n = 16, moments on the server)
-    "absmax": (8.012, "9f6de76b895cb432"),
-    "quantize": (12.150, "9f6de76b895cb432"),
-    "server": (26.52, "9f6de76b895cb432"),
+    # profiles/dram_traffic_flat28_n16_server_moments.txt: the benchmark's own workload
+    # (flat28, n = 16, moments on the server), one-pass capture of the two byte counters
+    "worker_fused": (20.05, "ada260155453a437"),
+    "server": (28.05, "ada260155453a437"),
 }
 
 

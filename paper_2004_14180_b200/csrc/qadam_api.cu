@@ -71,8 +71,8 @@ struct Geometry {
 // together with what phase 2 writes.
 size_t fused_group_bytes() {
   const char* env = std::getenv("QADAM_FUSED_GROUP_MB");
-  const long mb = env ? std::atol(env) : 24;
-  return (size_t)(mb > 0 ? mb : 24) << 20;
+  const long mb = env ? std::atol(env) : 20;
+  return (size_t)(mb > 0 ? mb : 20) << 20;
 }
 
 // Builds the run list of the fused worker kernel for all n workers.
@@ -129,7 +129,7 @@ void build_runs(const qadam_config* c, Geometry* g) {
   // from that (it sweeps L2 anyway): what is owed is finished before it, and it is
   // finished at once.
   const char* lag_env = std::getenv("QADAM_FUSED_LAG");
-  const int lag = std::max(1, lag_env ? std::atoi(lag_env) : 2);
+  const int lag = std::max(1, lag_env ? std::atoi(lag_env) : 1);
   std::vector<size_t> owed;                          // groups whose phase 2 is still to be emitted
   size_t owed_head = 0;
   for (size_t gi = 0; gi < groups.size(); ++gi) {
