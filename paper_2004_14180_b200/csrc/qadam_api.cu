@@ -303,19 +303,21 @@ ServerKernel pick_server(const qadam_ctx* c) {
 
 using PipeKernel = void (*)(const ServerParams, const CUtensorMap, const Tile*, int, int, int);
 
-template <bool SM>
+template <bool SM, int GB>
 PipeKernel pick_pipe_n(int n) {
   switch (n) {
-    case 4: return server_pipe_kernel<SM, 4>;
-    case 8: return server_pipe_kernel<SM, 8>;
-    case 16: return server_pipe_kernel<SM, 16>;
-    case 32: return server_pipe_kernel<SM, 32>;
-    default: return server_pipe_kernel<SM, 0>;
+    case 4: return server_pipe_kernel<SM, 4, GB>;
+    case 8: return server_pipe_kernel<SM, 8, GB>;
+    case 16: return server_pipe_kernel<SM, 16, GB>;
+    case 32: return server_pipe_kernel<SM, 32, GB>;
+    default: return server_pipe_kernel<SM, 0, GB>;
   }
 }
 
 PipeKernel pick_pipe(const qadam_ctx* c) {
-  return c->cfg.placement == QADAM_PLACE_SERVER ? pick_pipe_n<true>(c->cfg.n) : pick_pipe_n<false>(c->cfg.n);
+  const bool sm = c->cfg.placement == QADAM_PLACE_SERVER;
+  if (c->geo.gmode == G_FIVE) return sm ? pick_pipe_n<true, 3>(c->cfg.n) : pick_pipe_n<false, 3>(c->cfg.n);
+  return sm ? pick_pipe_n<true, 2>(c->cfg.n) : pick_pipe_n<false, 2>(c->cfg.n);
 }
 
 using WorkerPipeKernel = void (*)(const WorkerPipeParams, const int, const int);
@@ -463,7 +465,7 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
       !cuda_ok(cudaFuncSetAttribute(sk, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->server_smem))) {
     delete c; return QADAM_ERR_CUDA;
   }
-  // The pipelined server pass needs ternary codes, at most kPipeMaxWorkers streams and room
+  // The pipelined server pass needs ternary or five-level codes, at most kPipeMaxWorkers streams and room
   // for at least two stages in shared memory; otherwise the plain grid-stride kernel runs.
   {
     int max_smem = 0;
@@ -471,13 +473,15 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
       delete c; return QADAM_ERR_CUDA;
     }
     const bool sm_mom = cfg->placement == QADAM_PLACE_SERVER;
-    const size_t sb = pipe_stage_bytes(cfg->n, sm_mom);
+    const bool pipe_codes = c->geo.gmode == G_TERNARY || c->geo.gmode == G_FIVE;
+    const size_t sb = pipe_stage_bytes(cfg->n, sm_mom, pipe_codes ? c->geo.gbits : 2);
     const char* env = std::getenv("QADAM_SERVER_KERNEL");
     const bool want_plain = env && std::strcmp(env, "plain") == 0;
     int stages = (int)(((size_t)max_smem - 256) / sb);
     stages = pipe_legal_stages(std::min(stages, kPipeMaxStages));
-    if (!want_plain && c->geo.gmode == G_TERNARY && cfg->n <= kPipeMaxWorkers && stages >= 2 &&
-        make_codes_tensor_map(&c->codes_map, b->gcodes, (long long)c->geo.gcode_bytes, cfg->n)) {
+    if (!want_plain && pipe_codes && cfg->n <= kPipeMaxWorkers && stages >= 2 &&
+        make_codes_tensor_map(&c->codes_map, b->gcodes, (long long)c->geo.gcode_bytes, cfg->n,
+                              c->geo.gbits)) {
       c->pipe_stages = stages;
       c->pipe_smem = 256 + (size_t)stages * sb;
       if (!cuda_ok(cudaFuncSetAttribute(pick_pipe(c), cudaFuncAttributeMaxDynamicSharedMemorySize,

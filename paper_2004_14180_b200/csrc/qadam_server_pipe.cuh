@@ -1,7 +1,8 @@
-// The server pass for ternary codes as a persistent, warp-specialised pipeline.
+// The server pass for ternary and five-level codes as a persistent, warp-specialised
+// pipeline.
 //
 // One CTA per SM loops over 2048-element tiles.  A producer warp brings each
-// tile's inputs (x, m, v and the n workers' 512-byte code runs) into a ring of
+// tile's inputs (x, m, v and the n workers' code runs of 512 or 768 bytes) into a ring of
 // shared-memory stages with bulk asynchronous copies that complete on an
 // mbarrier; two groups of eight consumer warps take alternate tiles, decode,
 // average and update in place in shared memory and write the packed broadcast; a
@@ -114,12 +115,13 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsig
   return false;
 }
 
-// Tensor map over the n packed 2-bit code streams, seen as a 2-D array of 32-bit
-// words [n rows][gcode_bytes / 4], with a box of one tile's words (kPipeTile / 16)
-// by all n rows: one request brings every worker's codes of a tile, row after row,
+// Tensor map over the n packed code streams of gbits (2 or 3) bits per code, seen as a 2-D
+// array of 32-bit words [n rows][gcode_bytes / 4], with a box of one tile's words
+// (kPipeTile * gbits / 32) by all n rows: one request brings every worker's codes of a tile, row after row,
 // into shared memory.  Encoded through the driver entry point the runtime hands out,
 // so the library links against the runtime only.  Returns false if unavailable.
-inline bool make_codes_tensor_map(CUtensorMap* map, const void* gcodes, long long gcode_bytes, int n) {
+inline bool make_codes_tensor_map(CUtensorMap* map, const void* gcodes, long long gcode_bytes, int n,
+                                  int gbits) {
   typedef CUresult (*EncodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -131,7 +133,7 @@ inline bool make_codes_tensor_map(CUtensorMap* map, const void* gcodes, long lon
     return false;
   const cuuint64_t dims[2] = {(cuuint64_t)(gcode_bytes / 4), (cuuint64_t)n};
   const cuuint64_t strides[1] = {(cuuint64_t)gcode_bytes};          // bytes between rows
-  const cuuint32_t box[2] = {(cuuint32_t)(kPipeTile / 16), (cuuint32_t)n};
+  const cuuint32_t box[2] = {(cuuint32_t)(kPipeTile * gbits / 32), (cuuint32_t)n};
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = reinterpret_cast<EncodeTiled>(fn)(
       map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(gcodes), dims, strides, box, estr,
@@ -157,17 +159,17 @@ struct PipeSmem {
   int abort_flag;
 };
 
-// A stage: [header 128 B][x tile][m tile][v tile][n code runs of 512 B][n scales, each stored twice]
+// A stage: [header 128 B][x tile][m tile][v tile][n code runs of 256 * gbits B][n scales, each stored twice]
 struct StageHeader {
   long long off;   // first element of the tile
   int count;       // its length (multiple of 128, at most kPipeTile)
-  int pad;
+  int tiny;        // five-level codes: some scale is so small that half of it may not be a float
 };
 constexpr int kStageHeaderBytes = 128;
 
-__host__ __device__ inline size_t pipe_stage_bytes(int n, bool server_moments) {
+__host__ __device__ inline size_t pipe_stage_bytes(int n, bool server_moments, int gbits) {
   const size_t state = (server_moments ? 3 : 1) * (size_t)kPipeTile * sizeof(float);
-  const size_t codes = (size_t)n * (kPipeTile / 4);
+  const size_t codes = (size_t)n * (kPipeTile * gbits / 8);
   const size_t scales = ((size_t)n * 2 * sizeof(float) + 127) / 128 * 128;
   return kStageHeaderBytes + state + codes + scales;
 }
@@ -221,6 +223,72 @@ __device__ __forceinline__ void decode_accumulate(float2 sc, unsigned b0, unsign
   a[3] = fma2_rn(code_pair_minus_bias<0x30u, 0xc0u>(b1, mg[2], mg[3], k23), sc, a[3]);
 }
 
+// The same for 3-bit codes of the five-level grid {0, 1/2, 1} (code = level index + 2).
+// A lane's four codes of a row are 12 bits that start at bit 0 (even lanes) or bit 4 (odd
+// lanes) of a 16-bit window, so masks and exponents differ between lanes and sit in
+// registers.  The exponent gives a code's lowest bit the weight 1/2: the float reads
+// 2^E + code / 2, and subtracting 2^E + 1 leaves the level value (-1, -1/2, 0, 1/2, 1).
+struct FiveLevelLane {
+  unsigned mask[4];   // 7 << position of code c
+  unsigned mg[4];     // bit pattern of 2^E, E = 22 - position
+  float2 k01, k23;    // -(2^E + 1) for codes 0, 1 and 2, 3
+  unsigned zero;      // the 12 bits of four level-0 codes, at the lane's position
+  unsigned field;     // the lane's 12 bits
+};
+__device__ __forceinline__ FiveLevelLane five_level_lane(int lane) {
+  FiveLevelLane f;
+  const int sh = 4 * (lane & 1);
+  float kk[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const int pos = sh + 3 * c;
+    f.mask[c] = 7u << pos;
+    f.mg[c] = (unsigned)(149 - pos) << 23;
+    kk[c] = -(exp2i(22 - pos) + 1.0f);
+  }
+  f.k01 = make_float2(kk[0], kk[1]);
+  f.k23 = make_float2(kk[2], kk[3]);
+  f.zero = 0x492u << sh;
+  f.field = 0xfffu << sh;
+  return f;
+}
+__device__ __forceinline__ float2 level_pair(unsigned w, unsigned m_lo, unsigned mg_lo, unsigned m_hi,
+                                             unsigned mg_hi, float2 k) {
+  unsigned long long r;
+  asm("{\n\t.reg .b32 lo, hi;\n\t.reg .b64 t;\n\t"
+      "lop3.b32 lo, %1, %2, %3, 0xEA;\n\t"
+      "lop3.b32 hi, %1, %4, %5, 0xEA;\n\t"
+      "mov.b64 t, {lo, hi};\n\t"
+      "add.rn.f32x2 %0, t, %6;\n\t}"
+      : "=l"(r)
+      : "r"(w), "r"(m_lo), "r"(mg_lo), "r"(m_hi), "r"(mg_hi), "l"(pack_f2(k)));
+  return unpack_f2(r);
+}
+// One worker's contribution from its 16-bit windows w0, w1 of the tile's two rows.
+// EXACT = false: fma(level, scale, sum); the product is exact unless scale / 2 is not a
+// float, which the producer rules out per tile.  EXACT = true: the product is rounded
+// first, then added (scalar adds: a packed product feeding a packed add would be fused).
+template <bool EXACT>
+__device__ __forceinline__ void decode_accumulate5(float2 sc, unsigned w0, unsigned w1,
+                                                   const FiveLevelLane& f, float2 (&a)[4]) {
+  const float2 l0 = level_pair(w0, f.mask[0], f.mg[0], f.mask[1], f.mg[1], f.k01);
+  const float2 l1 = level_pair(w0, f.mask[2], f.mg[2], f.mask[3], f.mg[3], f.k23);
+  const float2 l2 = level_pair(w1, f.mask[0], f.mg[0], f.mask[1], f.mg[1], f.k01);
+  const float2 l3 = level_pair(w1, f.mask[2], f.mg[2], f.mask[3], f.mg[3], f.k23);
+  if constexpr (EXACT) {
+    const float2 q0 = mul2_rn(l0, sc), q1 = mul2_rn(l1, sc), q2 = mul2_rn(l2, sc), q3 = mul2_rn(l3, sc);
+    a[0] = make_float2(__fadd_rn(a[0].x, q0.x), __fadd_rn(a[0].y, q0.y));
+    a[1] = make_float2(__fadd_rn(a[1].x, q1.x), __fadd_rn(a[1].y, q1.y));
+    a[2] = make_float2(__fadd_rn(a[2].x, q2.x), __fadd_rn(a[2].y, q2.y));
+    a[3] = make_float2(__fadd_rn(a[3].x, q3.x), __fadd_rn(a[3].y, q3.y));
+  } else {
+    a[0] = fma2_rn(l0, sc, a[0]);
+    a[1] = fma2_rn(l1, sc, a[1]);
+    a[2] = fma2_rn(l2, sc, a[2]);
+    a[3] = fma2_rn(l3, sc, a[3]);
+  }
+}
+
 __device__ __forceinline__ unsigned opaque_u32(unsigned v) {
   unsigned r;
   asm volatile("mov.u32 %0, %1;" : "=r"(r) : "r"(v));
@@ -229,7 +297,8 @@ __device__ __forceinline__ unsigned opaque_u32(unsigned v) {
 
 // NW > 0: the worker count, known at compile time (the decode loop is unrolled and
 // every shared-memory offset is an immediate).  NW = 0: p.n workers, run-time loop.
-template <bool SERVER_MOMENTS, int NW>
+// GB: bits per gradient code, 2 (ternary) or 3 (five levels).
+template <bool SERVER_MOMENTS, int NW, int GB>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap codes_map,
                    const Tile* __restrict__ ptiles, const int num_ptiles, const int stages,
@@ -238,10 +307,13 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
   PipeSmem* ps = reinterpret_cast<PipeSmem*>(smem_raw);
   unsigned char* stage_base = smem_raw + 256;
   const int n = NW > 0 ? NW : p.n;
-  const unsigned stage_bytes = (unsigned)pipe_stage_bytes(n, SERVER_MOMENTS);
+  static_assert(GB == 2 || GB == 3, "code widths of the pipelined decode");
+  const unsigned stage_bytes = (unsigned)pipe_stage_bytes(n, SERVER_MOMENTS, GB);
   constexpr int kState = SERVER_MOMENTS ? 3 : 1;
   constexpr unsigned kCodesOff = kStageHeaderBytes + kState * kPipeTile * 4;
-  const unsigned scales_off = kCodesOff + (unsigned)n * (kPipeTile / 4);
+  constexpr int kRunBytes = kPipeTile * GB / 8;          // one worker's codes of a tile
+  constexpr int kRowBytes = kRunBytes / 2;               // of one of its two 1024-element rows
+  const unsigned scales_off = kCodesOff + (unsigned)n * kRunBytes;
   const int tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
 
@@ -265,6 +337,7 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
     // ------------------------------------------------------------------ producer
     int cur_seg = -1;
     float sc0 = 0.0f, sc1 = 0.0f;                       // scales of workers lane, lane + 32
+    int tiny = 0;
     int s = 0;
     unsigned ph = 0;
     int issued = 0;
@@ -277,6 +350,13 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
         cur_seg = t.seg;
         if (lane < n) sc0 = p.scales[(long long)lane * p.S + t.seg];
         if (lane + 32 < n) sc1 = p.scales[(long long)(lane + 32) * p.S + t.seg];
+        if (GB == 3) {
+          // half of a scale below 2^-120 may fall between floats; such a segment is summed
+          // with a rounded product instead of a fused one
+          const float lim = exp2i(-120);
+          tiny = __any_sync(0xffffffffu, (lane < n && sc0 != 0.0f && sc0 < lim) ||
+                                             (lane + 32 < n && sc1 != 0.0f && sc1 < lim));
+        }
       }
       // a fresh barrier passes a wait on the parity opposite to its first phase
       bool ok = true;
@@ -291,21 +371,22 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
         StageHeader* hd = reinterpret_cast<StageHeader*>(st);
         hd->off = t.off;
         hd->count = t.count;
+        hd->tiny = tiny;
       }
       __syncwarp();
       // one elected lane issues the tile's four requests: x, m, v runs and the code box.
-      // The box always carries n full 512-byte rows (beyond a short tile's length it holds
+      // The box always carries n full rows of kRunBytes (beyond a short tile's length it holds
       // the neighbouring codes or zero fill, which nobody reads).
       if (lane == 0) {
         const unsigned fbytes = (unsigned)t.count * 4u;
-        mbar_arrive_expect_tx(&ps->full[s], kState * fbytes + (unsigned)n * (kPipeTile / 4));
+        mbar_arrive_expect_tx(&ps->full[s], kState * fbytes + (unsigned)n * kRunBytes);
         float* sx = reinterpret_cast<float*>(st + kStageHeaderBytes);
         bulk_load(sx, p.x + t.off, fbytes, &ps->full[s]);
         if (SERVER_MOMENTS) {
           bulk_load(sx + kPipeTile, p.m + t.off, fbytes, &ps->full[s]);
           bulk_load(sx + 2 * kPipeTile, p.v + t.off, fbytes, &ps->full[s]);
         }
-        tensor_load_2d(st + kCodesOff, &codes_map, (int)(t.off >> 4), 0, &ps->full[s]);
+        tensor_load_2d(st + kCodesOff, &codes_map, (int)(t.off >> 5) * GB, 0, &ps->full[s]);
       }
       ++issued;
       if (++s == stages) { s = 0; ph ^= 1u; }
@@ -366,6 +447,9 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
     const float2 k23 = make_float2(-(exp2i(19) + 1.0f), -(exp2i(17) + 1.0f));
     const unsigned mg[4] = {opaque_u32(150u << 23), opaque_u32(148u << 23), opaque_u32(146u << 23),
                             opaque_u32(144u << 23)};
+    const FiveLevelLane fl = five_level_lane(lane);          // used by the 3-bit decode only
+    // the 3-bit decode holds more per worker in registers: unroll it by 8 at most
+    constexpr int kUnroll = NW > 0 ? (GB == 3 && NW > 8 ? 8 : NW) : 1;
     bool sparse_mode = true;          // warp-uniform: look for workers with nothing but level 0
     int dense_tiles_left = 0;
     int dense_span = 8;
@@ -379,33 +463,55 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
         const bool act1 = kPipeTile / 2 + gt * 4 < hd.count;
         if (act0) {
           float* sx = reinterpret_cast<float*>(st + kStageHeaderBytes) + gt * 4;
-          const unsigned char* s_codes = st + kCodesOff + gt;
+          // ternary: the thread's byte of a row; five levels: the first of its two bytes
+          const unsigned char* s_codes =
+              st + kCodesOff + (GB == 2 ? gt : gwarp * (128 * GB / 8) + ((lane * 3) >> 1));
+          const bool tiny = GB == 3 && hd.tiny != 0;
           const float2* s_scale = reinterpret_cast<const float2*>(st + scales_off);
           float2 a[4];
 #pragma unroll
           for (int c = 0; c < 4; ++c) a[c] = make_float2(0.0f, 0.0f);
-          // Zero skipping.  With a max-abs scale most ternary codes are level 0 (code 1,
-          // byte 0x55 for four of them), and a worker whose 256 codes in this warp's two
-          // rows are all level 0 adds +0 to every sum, which changes nothing (a sum is
-          // never -0).  The warp first votes, worker by worker and without branching, on
+          // Zero skipping.  With a max-abs scale most codes are level 0 (ternary: code 1,
+          // byte 0x55 for four of them; five levels: code 2), and a worker whose 256 codes
+          // in this warp's two rows are all level 0 adds +0 to every sum, which changes
+          // nothing (a sum is never -0).  The warp first votes, worker by worker and without branching, on
           // whether any lane holds a code other than 1, then decodes only the workers that
           // do, in increasing worker order (the order of the sum is unchanged).  When
           // more than an eighth of the workers have something to add the warp stops
           // looking for a while: the votes cost about half a decode, so denser codes are
           // decoded faster without them.
+          auto window = [&](int i, int r) -> unsigned {       // 3-bit codes: the lane's 16-bit window
+            const unsigned char* q = s_codes + i * kRunBytes + r * kRowBytes;
+            return (unsigned)q[0] | ((unsigned)q[1] << 8);
+          };
           auto contribute = [&](int i) {
-            decode_accumulate(s_scale[i], s_codes[i * (kPipeTile / 4)],
-                              s_codes[i * (kPipeTile / 4) + kPipeTile / 8], k01, k23, mg, a);
+            if constexpr (GB == 2) {
+              decode_accumulate(s_scale[i], s_codes[i * kRunBytes], s_codes[i * kRunBytes + kRowBytes], k01,
+                                k23, mg, a);
+            } else {
+              decode_accumulate5<false>(s_scale[i], window(i, 0), window(i, 1), fl, a);
+            }
           };
           auto has_nonzero = [&](int i) -> unsigned long long {
-            const unsigned b0 = s_codes[i * (kPipeTile / 4)];
-            const unsigned b1 = s_codes[i * (kPipeTile / 4) + kPipeTile / 8];
-            return __any_sync(0xffffffffu, (b0 & b1 & 0x55u) != 0x55u) ? 1ull : 0ull;
+            bool nz;
+            if constexpr (GB == 2) {
+              const unsigned b0 = s_codes[i * kRunBytes];
+              const unsigned b1 = s_codes[i * kRunBytes + kRowBytes];
+              nz = (b0 & b1 & 0x55u) != 0x55u;
+            } else {
+              nz = (((window(i, 0) ^ fl.zero) | (window(i, 1) ^ fl.zero)) & fl.field) != 0u;
+            }
+            return __any_sync(0xffffffffu, nz) ? 1ull : 0ull;
           };
-          if (sparse_mode) {
+          if (tiny) {
+            // rare: every worker, products rounded before they are added
+#pragma unroll 1
+            for (int i = 0; i < n; ++i)
+              decode_accumulate5<true>(s_scale[i], window(i, 0), window(i, 1), fl, a);
+          } else if (sparse_mode) {
             unsigned long long live = 0;
             if constexpr (NW > 0) {
-#pragma unroll
+#pragma unroll kUnroll
               for (int i = 0; i < NW; ++i) live |= has_nonzero(i) << i;
             } else {
 #pragma unroll 4
@@ -427,7 +533,7 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
             }
           } else {
             if constexpr (NW > 0) {
-#pragma unroll
+#pragma unroll kUnroll
               for (int i = 0; i < NW; ++i) contribute(i);
             } else {
 #pragma unroll 4

@@ -142,6 +142,54 @@ def test_sparse_and_dense_code_regions(placement):
     p.close()
 
 
+@pytest.mark.parametrize("n", [1, 4, 8, 16, 32, 33, 64])
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_five_level_worker_counts(n, placement):
+    # 3-bit codes through the pipelined server pass: unrolled (4, 8, 16, 32) and run-time worker loops
+    _run([6000, 300, 3 * 2048 + 128], n, 1, 1, placement, T=2, seed=200 + n)
+
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_five_level_scales_whose_half_is_not_a_float(placement):
+    """Five-level codes decode to scale / 2 for the inner levels.  With every scale a
+    small odd multiple of the smallest subnormal that product is rounded before it is
+    added (Section 5.1 defines the decoded value, the sum comes after), which a fused
+    multiply-add would not reproduce; one ordinary segment rides along."""
+    rng = np.random.default_rng(31)
+    seg, n = [4096 + 128, 2048], 5
+    d = sum(seg)
+    p = Pair(seg, n, 1, 0, placement, x1=np.zeros(d, np.float32))
+    tiny = np.float32(2.0 ** -149)
+    for t in range(3):
+        g = np.zeros((n, d), np.float32)
+        k = rng.integers(-7, 8, (n, seg[0])).astype(np.float32)
+        k[:, t] = np.array([7, 5, 7, 3, 5], np.float32)          # odd maxima
+        g[:, :seg[0]] = k * tiny
+        g[:, seg[0]:] = (rng.standard_normal((n, seg[1])) * 0.01).astype(np.float32)
+        p.step(g)
+        p.compare_state()
+    p.close()
+
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_five_level_sparse_and_dense_code_regions(placement):
+    rng = np.random.default_rng(78)
+    d, n = 1 << 23, 8
+    dense_end = d * 3 // 10
+    x1 = (rng.standard_normal(d) * 0.05).astype(np.float32)
+    p = Pair([d], n, 1, 0, placement, x1=x1)
+    for t in range(2):
+        g = (rng.standard_normal((n, d)) * 1e-4).astype(np.float32)
+        g[:, :dense_end] = rng.standard_normal((n, dense_end)).astype(np.float32)
+        hits = rng.integers(dense_end, d, (n, 300))
+        for i in range(n):
+            g[i, hits[i]] = rng.choice(np.array([4.0, -4.0, 2.0, -2.0], np.float32), 300)
+        g[:, d - 1] = 5.0
+        p.step(g, threads=4)
+    p.compare_state()
+    p.close()
+
+
 def test_nonfinite_input_sets_status_bit():
     import paper_2004_14180_b200 as qb
     q = qb.QAdam([1000], 1, kg=0, kx=-1)
