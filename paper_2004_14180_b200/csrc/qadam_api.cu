@@ -241,6 +241,7 @@ struct qadam_ctx {
   size_t server_smem;
   // persistent pipelined server pass (ternary codes): stages > 0 when in use
   int pipe_stages = 0;
+  int pipe_skip_16ths = 2;   // zero skipping while at most this many sixteenths of the workers are live
   size_t pipe_smem = 0;
   CUtensorMap codes_map;
   // pipelined worker kernel (moments on the server, all workers in one call): grid > 0 when in use
@@ -301,7 +302,7 @@ ServerKernel pick_server(const qadam_ctx* c) {
   }
 }
 
-using PipeKernel = void (*)(const ServerParams, const CUtensorMap, const Tile*, int, int, int);
+using PipeKernel = void (*)(const ServerParams, const CUtensorMap, const Tile*, int, int, int, int);
 
 template <bool SM, int GB>
 PipeKernel pick_pipe_n(int n) {
@@ -483,6 +484,10 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
         make_codes_tensor_map(&c->codes_map, b->gcodes, (long long)c->geo.gcode_bytes, cfg->n,
                               c->geo.gbits)) {
       c->pipe_stages = stages;
+      if (const char* sk16 = std::getenv("QADAM_SKIP_16THS")) {
+        const int v = std::atoi(sk16);
+        if (v >= 0 && v <= 16) c->pipe_skip_16ths = v;
+      }
       c->pipe_smem = 256 + (size_t)stages * sb;
       if (!cuda_ok(cudaFuncSetAttribute(pick_pipe(c), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)c->pipe_smem))) {
@@ -647,7 +652,7 @@ int qadam_server_step(qadam_ctx* c, int64_t step, float lr_t) {
       const int np = (int)c->geo.ptiles.size();
       const int pgrid = std::min(c->sm_count, np);
       pick_pipe(c)<<<pgrid, kPipeThreads, c->pipe_smem, c->stream>>>(p, c->codes_map, c->d_ptiles, np,
-                                                                      c->pipe_stages, inv_exact);
+                                                                      c->pipe_stages, inv_exact, c->pipe_skip_16ths);
     } else {
       pick_server(c)<<<grid, kThreads, c->server_smem, c->stream>>>(p);
     }

@@ -302,7 +302,7 @@ template <bool SERVER_MOMENTS, int NW, int GB>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap codes_map,
                    const Tile* __restrict__ ptiles, const int num_ptiles, const int stages,
-                   const int inv_n_exact) {
+                   const int inv_n_exact, const int skip_16ths) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   PipeSmem* ps = reinterpret_cast<PipeSmem*>(smem_raw);
   unsigned char* stage_base = smem_raw + 256;
@@ -492,6 +492,21 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
               decode_accumulate5<false>(s_scale[i], window(i, 0), window(i, 1), fl, a);
             }
           };
+          auto contribute_pair = [&](int i0, int i1, bool two) {
+            const float2 sc0 = s_scale[i0];
+            const float2 sc1 = two ? s_scale[i1] : make_float2(0.0f, 0.0f);
+            if constexpr (GB == 2) {
+              const unsigned p0 = s_codes[i0 * kRunBytes], p1 = s_codes[i0 * kRunBytes + kRowBytes];
+              const unsigned q0 = s_codes[i1 * kRunBytes], q1 = s_codes[i1 * kRunBytes + kRowBytes];
+              decode_accumulate(sc0, p0, p1, k01, k23, mg, a);
+              decode_accumulate(sc1, q0, q1, k01, k23, mg, a);
+            } else {
+              const unsigned p0 = window(i0, 0), p1 = window(i0, 1);
+              const unsigned q0 = window(i1, 0), q1 = window(i1, 1);
+              decode_accumulate5<false>(sc0, p0, p1, fl, a);
+              decode_accumulate5<false>(sc1, q0, q1, fl, a);
+            }
+          };
           auto has_nonzero = [&](int i) -> unsigned long long {
             bool nz;
             if constexpr (GB == 2) {
@@ -517,7 +532,7 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
 #pragma unroll 4
               for (int i = 0; i < n; ++i) live |= has_nonzero(i) << i;
             }
-            if (8 * __popcll(live) > n) {
+            if (16 * __popcll(live) > skip_16ths * n) {
               // too many live workers for the vote to pay: decode everything for a while,
               // looking again after 16, 32, ... up to 1024 tiles
               sparse_mode = false;
@@ -526,10 +541,15 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
             } else {
               dense_span = 8;
             }
+            // live workers two at a time, so that the loads and the bit work of one overlap
+            // the other's; an odd one out is paired with scale 0, which adds nothing
             while (live) {
-              const int i = __ffsll((long long)live) - 1;
+              const int i0 = __ffsll((long long)live) - 1;
               live &= live - 1;
-              contribute(i);
+              const bool two = live != 0;
+              const int i1 = two ? __ffsll((long long)live) - 1 : i0;
+              live &= live - 1;
+              contribute_pair(i0, i1, two);
             }
           } else {
             if constexpr (NW > 0) {
