@@ -46,6 +46,7 @@ class _Problem(C.Structure):
         ("seg_len", C.POINTER(C.c_int64)), ("seg_off", C.POINTER(C.c_int64)),
         ("kg", C.c_int32), ("kx", C.c_int32), ("grid_g", C.c_int32), ("placement", C.c_int32),
         ("beta", C.c_float), ("theta", C.c_float), ("eps", C.c_float),
+        ("weight_decay", C.c_float),
     ]
 
 
@@ -81,7 +82,7 @@ def lib():
         L.qo_unpack_bits.restype = None
         L.qo_unpack_bits.argtypes = [u8p, C.c_int64, C.c_int32, u32p]
         L.qo_worker_step.restype = C.c_int32
-        L.qo_worker_step.argtypes = [pp, f32p, f32p, f32p, f32p, C.c_float, f32p, u8p]
+        L.qo_worker_step.argtypes = [pp, f32p, f32p, f32p, f32p, f32p, C.c_float, f32p, u8p]
         L.qo_broadcast_weights.restype = C.c_int32
         L.qo_broadcast_weights.argtypes = [pp, f32p, u8p, f32p]
         L.qo_server_step.restype = C.c_int32
@@ -185,7 +186,7 @@ class OracleState:
         self.kg, self.kx, self.grid_g, self.placement = kg, kx, grid_g, placement
         self._prob = _Problem(self.d, self.D, self.n, self.S,
                               _p(self.seg_len, C.c_int64), _p(self.seg_off, C.c_int64),
-                              kg, kx, grid_g, placement, beta1, beta2, eps)
+                              kg, kx, grid_g, placement, beta1, beta2, eps, 0.0)
         self.gcode_bytes = int(lib().qo_gcode_bytes(C.byref(self._prob)))
         self.wcode_bytes = int(lib().qo_wcode_bytes(C.byref(self._prob)))
         D = self.D
@@ -228,13 +229,30 @@ class OracleState:
                                    _p(self.wcodes, C.c_uint8) if self.kx >= 0 else None,
                                    _p(self.wresid, C.c_float))
 
+    # step-dependent parameters -------------------------------------------------
+    def set_moment_rates(self, beta_t: float, theta_t: float) -> None:
+        """beta_t, theta_t of Algorithm 1 for the steps that follow."""
+        self._prob.beta, self._prob.theta = beta_t, theta_t
+
+    def set_regularization(self, weight_decay: float) -> None:
+        """lambda of the l2 term (Section 5.1) for the steps that follow."""
+        self._prob.weight_decay = weight_decay
+        self._xhat = None
+
+    def held_weights(self) -> np.ndarray:
+        """What the workers hold during a step: the decoded broadcast, or x itself
+        when the weights are not quantized."""
+        return self.decoded_weights() if self.kx >= 0 else self.x
+
     # steps -------------------------------------------------------------------
-    def worker_step(self, i: int, g_padded: np.ndarray, lr: float) -> None:
+    def worker_step(self, i: int, g_padded: np.ndarray, lr: float, xhat: np.ndarray = None) -> None:
         g = np.ascontiguousarray(g_padded, dtype=np.float32)
         assert g.shape == (self.D,)
         wm = self.placement == PLACE_WORKER
+        if xhat is None and self._prob.weight_decay != 0.0:
+            xhat = self.held_weights()
         rc = lib().qo_worker_step(
-            C.byref(self._prob), _p(g, C.c_float),
+            C.byref(self._prob), _p(g, C.c_float), _p(xhat, C.c_float),
             _p(self.m[i], C.c_float) if wm else None,
             _p(self.v[i], C.c_float) if wm else None,
             _p(self.e[i], C.c_float), lr,
@@ -246,12 +264,13 @@ class OracleState:
         """All n workers.  The oracle itself is single-threaded; `threads` > 1
         only runs independent workers side by side."""
         assert g_padded.shape == (self.n, self.D)
+        xhat = self.held_weights() if self._prob.weight_decay != 0.0 else None
         if threads <= 1:
             for i in range(self.n):
-                self.worker_step(i, g_padded[i], lr)
+                self.worker_step(i, g_padded[i], lr, xhat)
         else:
             with ThreadPoolExecutor(max_workers=threads) as ex:
-                list(ex.map(lambda i: self.worker_step(i, g_padded[i], lr), range(self.n)))
+                list(ex.map(lambda i: self.worker_step(i, g_padded[i], lr, xhat), range(self.n)))
 
     def server_step(self, lr: float) -> None:
         sm = self.placement == PLACE_SERVER

@@ -234,7 +234,9 @@ typedef struct {
   int32_t kx;                // -1: Q_x = identity (nothing broadcast in packed form)
   int32_t grid_g;            // 0 POW2, 1 UNIFORM
   int32_t placement;         // where m, v live
-  float beta, theta, eps;
+  float beta, theta, eps;    // beta_t, theta_t of the step at hand (the caller may change them
+                             // between steps: Assumption 2's theta_t = 1 - theta/t)
+  float weight_decay;        // lambda of the l2 term (Section 5.1); 0: none
 } qo_problem;
 
 // Padded layout: segment s starts at the next multiple of 128 elements.
@@ -308,12 +310,14 @@ void qo_unpack_bits(const uint8_t* in, int64_t count, int32_t bits, uint32_t* co
 //   contrasts with): u = g + e, moments are the server's.
 // READING (identity Q_g): the stream is the raw binary32 of u, scale 1, e = 0.
 // ---------------------------------------------------------------------------
-int32_t qo_worker_step(const qo_problem* p, const float* g, float* m, float* v,
+int32_t qo_worker_step(const qo_problem* p, const float* g, const float* xhat, float* m, float* v,
                        float* e, float alpha, float* scales, uint8_t* codes) {
   const Hyper h = make_hyper(p->beta, p->theta, p->eps);
   GradLevels G;
   if (p->kg >= 0 && !make_grad_levels(p->kg, p->grid_g, &G)) return -1;
   if (p->placement == QO_PLACE_WORKER && (!m || !v)) return -2;
+  const float lambda = p->weight_decay;
+  if (lambda != 0.0f && !xhat) return -3;
 
   std::vector<float> u;
   std::vector<int32_t> q;
@@ -324,11 +328,19 @@ int32_t qo_worker_step(const qo_problem* p, const float* g, float* m, float* v,
     u.assign((size_t)len, 0.0f);
     for (int64_t j = 0; j < len; ++j) {
       const int64_t k = off + j;
+      // READING (l2 term): "l2 regularization with a scalar 5e-4 as the weight decay term"
+      // (Section 5.1) adds lambda/2 |x|^2 to each worker's loss, i.e. lambda times the weight
+      // the worker holds, which is the broadcast Q_x(x_t), to its stochastic gradient.
+      float gk = g[k];
+      if (lambda != 0.0f) {
+        const float term = lambda * xhat[k];
+        gk = gk + term;
+      }
       if (p->placement == QO_PLACE_WORKER) {
-        moments(h, g[k], &m[k], &v[k]);
+        moments(h, gk, &m[k], &v[k]);
         u[j] = adam_step(h, m[k], v[k], alpha) + e[k];
       } else {
-        u[j] = g[k] + e[k];
+        u[j] = gk + e[k];
       }
     }
     if (p->kg < 0) {
