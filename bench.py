@@ -43,8 +43,9 @@ NCU_TRAFFIC = {
     # kernel: (bytes per unit, digest of csrc/ at capture time)
     # profiles/dram_traffic_flat28_n16_server_moments.txt: the benchmark's own workload
     # (flat28, n = 16, moments on the server), one-pass capture of the two byte counters
-    "worker_fused": (20.05, "ada260155453a437"),
-    "server": (28.05, "ada260155453a437"),
+    "absmax": (8.00, "8cd9bfdcf5c36862"),
+    "quantize": (12.24, "8cd9bfdcf5c36862"),
+    "server": (28.03, "8cd9bfdcf5c36862"),
 }
 
 
@@ -71,6 +72,8 @@ def parse_args():
     ap.add_argument("--kg", type=int, default=None)
     ap.add_argument("--kx", type=int, default=None)
     ap.add_argument("--single-scale", action="store_true", help="one max-abs scale per worker")
+    ap.add_argument("--weight-decay", type=float, default=0.0,
+                    help="lambda of the l2 term g + lambda * (held weights); 0: none")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -150,7 +153,7 @@ class ClockSampler:
 # ----------------------------------------------------------------------------- byte accounting
 
 def algorithmic_bytes(kernel: str, w, placement: str, D: int, gbits: int, xbits: int,
-                      pass_model=None) -> float:
+                      pass_model=None, l2_term: bool = False) -> float:
     """Bytes one launch of `kernel` must move at its interface (fp32 state it has
     to read and write, packed codes), for all n workers.  For the fused worker kernel
     the figure is capacity aware: (worker, segment) pairs that fit the kernel's L2
@@ -158,6 +161,8 @@ def algorithmic_bytes(kernel: str, w, placement: str, D: int, gbits: int, xbits:
     needs the whole pair before any of it can be quantized)."""
     n = w.n
     server_moments = placement == "server"
+    # with the l2 term a worker also reads the weights it holds: the packed broadcast, or x
+    held = ((xbits / 8.0) if xbits else 4.0) if l2_term else 0.0
     if kernel == "worker_fused":
         one_pass, two_pass = pass_model
         if server_moments:      # read g, e (twice when two-pass); write e and the codes
@@ -165,13 +170,13 @@ def algorithmic_bytes(kernel: str, w, placement: str, D: int, gbits: int, xbits:
         # read g, m, v, e; write m, v, e and codes; two-pass adds a write and a read of u
         return one_pass * (28.0 + gbits / 8.0) + two_pass * (36.0 + gbits / 8.0)
     if kernel == "absmax":      # phase 1: read g, e (worker moments: + read m, v, write m, v, u)
-        per = 8.0 if server_moments else 28.0
+        per = (8.0 if server_moments else 28.0) + held
         return per * n * D
     if kernel == "quantize":    # phase 2: read g, e (or u), write e and the codes
-        per = (12.0 if server_moments else 8.0) + gbits / 8.0
+        per = (12.0 + held if server_moments else 8.0) + gbits / 8.0
         return per * n * D
     if kernel == "identity":
-        per = (8.0 + 8.0) if server_moments else (16.0 + 16.0)
+        per = ((8.0 + 8.0) if server_moments else (16.0 + 16.0)) + held
         return per * n * D
     if kernel == "server":      # read n code streams and x (m, v); write x (m, v) and the broadcast
         state = 24.0 if server_moments else 8.0
@@ -183,7 +188,7 @@ def algorithmic_bytes(kernel: str, w, placement: str, D: int, gbits: int, xbits:
 
 # ----------------------------------------------------------------------------- the oracle, timed
 
-def time_oracle(w, placement: str, sample_log2: int, steps: int, warmup: int):
+def time_oracle(w, placement: str, sample_log2: int, steps: int, warmup: int, weight_decay: float = 0.0):
     """Times the CPU oracle (single thread) on a bounded sample of the workload:
     the same n, quantizers and distributions, each worker's vector cut to
     2**sample_log2 elements.  Returns (elements/s, description, seconds per step)."""
@@ -198,6 +203,7 @@ def time_oracle(w, placement: str, sample_log2: int, steps: int, warmup: int):
     place = oracle.PLACE_SERVER if placement == "server" else oracle.PLACE_WORKER
     st = oracle.OracleState([d_s], ws.n, ws.kg, ws.kx, place, ws.beta1, ws.beta2, ws.eps)
     st.set_weights(qi.initial_weights(ws, "cpu").numpy())
+    st.set_regularization(weight_decay)
     g = st.to_padded(np.stack([qi.gradients(ws, 1, i, "cpu").numpy() for i in range(ws.n)]))
     for _ in range(warmup):
         st.step(g, ws.lr, threads=1)
@@ -216,7 +222,7 @@ def run_reference(args):
         return
     w = get_workload(args)
     sample_log2 = args.sample_log2 or 22
-    value, desc, dt = time_oracle(w, args.placement, sample_log2, args.steps, args.warmup)
+    value, desc, dt = time_oracle(w, args.placement, sample_log2, args.steps, args.warmup, args.weight_decay)
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT,
         "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
@@ -234,7 +240,7 @@ def workload_config(w, args, extra=None):
     cfg = {
         "workload": f"{w.name} (d={w.d}, {w.num_segments} scale segment(s), n={w.n} workers)",
         "d": w.d, "n_workers": w.n, "segments": w.num_segments,
-        "kg": w.kg, "kx": w.kx, "placement": args.placement,
+        "kg": w.kg, "kx": w.kx, "placement": args.placement, "weight_decay": args.weight_decay,
         "beta1": w.beta1, "beta2": w.beta2, "eps": w.eps, "lr": w.lr,
         "gradients": w.grad, "parallelism": f"replicas x{args.gpus} (no exchange between GPUs)",
         "l2": ("inputs larger than L2 (no flush between steps)" if 8 * w.n * w.d > (1 << 28) else
@@ -291,6 +297,7 @@ def run_b200(args):
     x1 = qi.initial_weights(w, dev)
     q = qb.QAdam(w.scale_seg_len, w.n, kg=w.kg, kx=w.kx, placement=placement, beta1=w.beta1,
                  beta2=w.beta2, eps=w.eps, lr=w.lr, x1=x1, device=dev)
+    q.set_regularization(args.weight_decay)
     del x1
     D = q.D
     if w.n * D * 4 <= (1 << 27):
@@ -371,7 +378,7 @@ def run_b200(args):
             continue
         per = ms / cnt
         bytes_ = algorithmic_bytes(name, w, args.placement, D, q.gcode_bytes * 8 // D, q.wcode_bytes * 8 // D,
-                                   pass_model=q.worker_pass_model())
+                                   pass_model=q.worker_pass_model(), l2_term=args.weight_decay != 0.0)
         kernels[name] = {"launches": int(cnt), "ms_per_launch": per,
                          "share": ms / sum(m for m, c in prof.values()),
                          "algorithmic_bytes": bytes_, "achieved_gbs": bytes_ / (per * 1e-3) / 1e9,
@@ -391,7 +398,7 @@ def run_b200(args):
         cpu_baseline = None
         if not args.no_cpu_baseline and world == 1:
             sl = args.sample_log2 or 24
-            v, desc, _ = time_oracle(w, args.placement, sl, steps=2, warmup=0)
+            v, desc, _ = time_oracle(w, args.placement, sl, steps=2, warmup=0, weight_decay=args.weight_decay)
             cpu_baseline = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
         sent = q.sent_bytes_per_step()
         line = {

@@ -171,6 +171,23 @@ int qadam_server_step(qadam_ctx* ctx, int64_t step, float lr_t);
 int qadam_step_host(qadam_ctx* ctx, int64_t step, const float* g_host, float* g_stage,
                     void* out_host, float lr_t);
 
+/* Algorithm 1's step-dependent rates: beta_t and theta_t used by every later call (the
+ * moments are updated by the workers under PLACE_WORKER and by the server under
+ * PLACE_SERVER, so call it between steps, not between a step's worker and server
+ * halves).  The caller computes the schedule, e.g. Assumption 2's theta_t = 1 - theta/t
+ * with beta_t in [0, beta]; the base learning rate alpha_t = alpha/sqrt(t) is each call's
+ * lr_t.  Host call, nothing is enqueued.  0 <= beta_t < 1 and 0 <= theta_t < 1, else
+ * QADAM_ERR_HYPER and nothing changes. */
+int qadam_set_moment_rates(qadam_ctx* ctx, float beta_t, float theta_t);
+
+/* The l2 term of Section 5.1 ("l2 regularization with a scalar 5e-4 as the weight decay
+ * term"): every later qadam_worker_compress uses g + lambda * w in place of g, where w is
+ * the weight vector the workers hold during the step: the broadcast Q_x(x_t) decoded from
+ * wcodes (kx >= 0), or x itself (kx = -1).  Rounded as fl(g + fl(lambda * w)).  lambda = 0
+ * (the state after qadam_create) switches the term off.  Host call, nothing is enqueued.
+ * lambda must be finite and >= 0, else QADAM_ERR_HYPER. */
+int qadam_set_regularization(qadam_ctx* ctx, float lambda);
+
 /* Worker scales without any allocation (no counterpart in the paper: a service
  * entry point for callers that cannot allocate device memory at all, such as a
  * process that sizes its device memory once at start-up and forbids cudaMalloc

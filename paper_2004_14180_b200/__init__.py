@@ -14,6 +14,6 @@ from .binding import (  # noqa: F401
     qadam_query_sizes, qadam_grad_code_bits, qadam_weight_code_bits,
     qadam_create, qadam_worker_compress, qadam_server_step, qadam_step_host,
     qadam_worker_scales_static, STATIC_MAX_ELEMENTS, STATIC_MAX_WORKERS,
-    qadam_worker_pass_model,
+    qadam_worker_pass_model, qadam_set_moment_rates, qadam_set_regularization,
     qadam_poll_status, qadam_profile_enable, qadam_profile_read, KERNEL_NAMES, qadam_launch_count, qadam_destroy, qadam_strerror,
 )

@@ -24,7 +24,7 @@ exported_symbols = (
     "qadam_worker_compress", "qadam_server_step", "qadam_step_host", "qadam_poll_status",
     "qadam_launch_count", "qadam_destroy", "qadam_strerror", "qadam_last_cuda_error",
     "qadam_profile_enable", "qadam_profile_read", "qadam_worker_scales_static",
-    "qadam_worker_pass_model",
+    "qadam_worker_pass_model", "qadam_set_moment_rates", "qadam_set_regularization",
 )
 
 STATIC_MAX_ELEMENTS = 1 << 26
@@ -104,6 +104,10 @@ def load_library():
     L.qadam_worker_scales_static.argtypes = [C.c_void_p, C.c_void_p, C.c_int64, C.c_int32, C.c_void_p, C.c_void_p]
     L.qadam_worker_pass_model.restype = C.c_int
     L.qadam_worker_pass_model.argtypes = [C.c_void_p, C.POINTER(C.c_int64), C.POINTER(C.c_int64)]
+    L.qadam_set_moment_rates.restype = C.c_int
+    L.qadam_set_moment_rates.argtypes = [C.c_void_p, C.c_float, C.c_float]
+    L.qadam_set_regularization.restype = C.c_int
+    L.qadam_set_regularization.argtypes = [C.c_void_p, C.c_float]
     L.qadam_launch_count.restype = C.c_int64
     L.qadam_launch_count.argtypes = [C.c_void_p]
     L.qadam_destroy.restype = C.c_int
@@ -173,6 +177,14 @@ def qadam_poll_status(ctx: int) -> int:
     st = C.c_uint32()
     _check(load_library().qadam_poll_status(ctx, C.byref(st)), "qadam_poll_status")
     return st.value
+
+
+def qadam_set_moment_rates(ctx: int, beta_t: float, theta_t: float) -> None:
+    _check(load_library().qadam_set_moment_rates(ctx, beta_t, theta_t), "qadam_set_moment_rates")
+
+
+def qadam_set_regularization(ctx: int, weight_decay: float) -> None:
+    _check(load_library().qadam_set_regularization(ctx, weight_decay), "qadam_set_regularization")
 
 
 def qadam_profile_enable(ctx: int, enable: bool) -> None:
@@ -324,6 +336,14 @@ class QAdam:
 
     def poll_status(self) -> int:
         return qadam_poll_status(self.ctx)
+
+    def set_moment_rates(self, beta_t: float, theta_t: float) -> None:
+        """beta_t, theta_t of Algorithm 1 for the steps that follow."""
+        qadam_set_moment_rates(self.ctx, beta_t, theta_t)
+
+    def set_regularization(self, weight_decay: float) -> None:
+        """lambda of the l2 term (Section 5.1) for the steps that follow; 0 switches it off."""
+        qadam_set_regularization(self.ctx, weight_decay)
 
     @property
     def launches(self) -> int:

@@ -108,6 +108,10 @@ void build_runs(const qadam_config* c, Geometry* g) {
   }
   g->runs.clear();
   long long item = 0;
+  const char* sk_env = std::getenv("QADAM_SOLO_KEEP");
+  const char* sb_env = std::getenv("QADAM_SOLO_BACK");
+  const bool solo_keep = sk_env ? std::atoi(sk_env) != 0 : true;
+  const bool solo_back = sb_env ? std::atoi(sb_env) != 0 : true;
   auto emit = [&](size_t gi, int phase) {
     for (const Pair& pr : groups[gi]) {
       Run r;
@@ -118,7 +122,9 @@ void build_runs(const qadam_config* c, Geometry* g) {
       r.worker = pr.worker;
       r.seg = pr.seg;
       r.phase = phase;
-      r.dir = (phase == 1 && solo[gi]) ? -1 : 1;    // a lone big pair: phase 2 walks back over the cached tail
+      r.dir = (phase == 1 && solo[gi] && solo_back) ? -1 : 1;   // a lone big pair: phase 2 walks back over the cached tail
+      r.keep = (phase == 0 && (!solo[gi] || solo_keep)) ? 1 : 0;
+      r.pad = 0;
       g->runs.push_back(r);
       item += r.ntiles;
     }
@@ -240,6 +246,7 @@ struct qadam_ctx {
   int grid_absmax, grid_quant, grid_ident, grid_server, grid_bcast;
   size_t server_smem;
   // persistent pipelined server pass (ternary codes): stages > 0 when in use
+  float lambda = 0.0f;       // l2 term (qadam_set_regularization)
   int pipe_stages = 0;
   int pipe_skip_16ths = 2;   // zero skipping while at most this many sixteenths of the workers are live
   size_t pipe_smem = 0;
@@ -272,17 +279,28 @@ using WorkerKernel = void (*)(const WorkerParams);
 using ServerKernel = void (*)(const ServerParams);
 
 WorkerKernel pick_absmax(const qadam_ctx* c) {
-  return c->cfg.placement == QADAM_PLACE_WORKER ? worker_absmax_kernel<true>
-                                                : worker_absmax_kernel<false>;
+  const bool w = c->cfg.placement == QADAM_PLACE_WORKER;
+  if (c->lambda != 0.0f) return w ? worker_absmax_kernel<true, true> : worker_absmax_kernel<false, true>;
+  return w ? worker_absmax_kernel<true> : worker_absmax_kernel<false>;
 }
 
 WorkerKernel pick_identity(const qadam_ctx* c) {
-  return c->cfg.placement == QADAM_PLACE_WORKER ? worker_identity_kernel<true>
-                                                : worker_identity_kernel<false>;
+  const bool w = c->cfg.placement == QADAM_PLACE_WORKER;
+  if (c->lambda != 0.0f) return w ? worker_identity_kernel<true, true> : worker_identity_kernel<false, true>;
+  return w ? worker_identity_kernel<true> : worker_identity_kernel<false>;
 }
 
 WorkerKernel pick_quantize(const qadam_ctx* c) {
   const bool w = c->cfg.placement == QADAM_PLACE_WORKER;
+  if (!w && c->lambda != 0.0f) {
+    // moments on the server: phase 2 forms u = g + e again, l2 term included
+    switch (c->geo.gmode) {
+      case G_TERNARY: return worker_quantize_kernel<false, G_TERNARY, true>;
+      case G_FIVE:    return worker_quantize_kernel<false, G_FIVE, true>;
+      case G_POW2:    return worker_quantize_kernel<false, G_POW2, true>;
+      default:        return worker_quantize_kernel<false, G_UNIFORM, true>;
+    }
+  }
   switch (c->geo.gmode) {
     case G_TERNARY: return w ? worker_quantize_kernel<true, G_TERNARY> : worker_quantize_kernel<false, G_TERNARY>;
     case G_FIVE:    return w ? worker_quantize_kernel<true, G_FIVE>    : worker_quantize_kernel<false, G_FIVE>;
@@ -330,6 +348,13 @@ WorkerPipeKernel pick_worker_pipe(const qadam_ctx* c) {
     case G_POW2:    return worker_pipe_kernel<G_POW2>;
     default:        return worker_pipe_kernel<G_UNIFORM>;
   }
+}
+
+// grids of the split worker kernels (they depend on whether the l2 term is on)
+void plan_worker_grids(qadam_ctx* c) {
+  c->grid_absmax = resident_grid(pick_absmax(c), 0, c->sm_count);
+  c->grid_quant = resident_grid(pick_quantize(c), 0, c->sm_count);
+  c->grid_ident = resident_grid(pick_identity(c), 0, c->sm_count);
 }
 
 cudaEvent_t take_event(qadam_ctx* c) {
@@ -495,17 +520,19 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
       }
     }
   }
-  c->grid_absmax = resident_grid(pick_absmax(c), 0, c->sm_count);
-  c->grid_quant = resident_grid(pick_quantize(c), 0, c->sm_count);
-  c->grid_ident = resident_grid(pick_identity(c), 0, c->sm_count);
+  plan_worker_grids(c);
   c->grid_server = resident_grid(sk, c->server_smem, c->sm_count);
   c->grid_bcast = resident_grid(weight_broadcast_kernel, 0, c->sm_count);
   // The pipelined worker kernel needs every CTA resident at once (its phase-2 items wait
-  // for phase-1 items of other CTAs): one CTA per SM, launched cooperatively.
+  // for phase-1 items of other CTAs): one CTA per SM, launched cooperatively.  It pays
+  // through the (worker, segment) pairs that stay in L2 between the phases; when no pair
+  // does (every segment larger than a group) the two plain streaming launches are a few
+  // per cent faster (measured) and run instead, unless QADAM_WORKER_KERNEL=pipe.
   {
     int coop = 0, max_smem = 0;
     const char* env = std::getenv("QADAM_WORKER_KERNEL");
-    const bool want_split = env && std::strcmp(env, "split") == 0;
+    const bool want_split = (env && std::strcmp(env, "split") == 0) ||
+                            (c->geo.one_pass_elems == 0 && !(env && std::strcmp(env, "pipe") == 0));
     if (!want_split && c->geo.gmode != G_IDENTITY && cfg->placement == QADAM_PLACE_SERVER &&
         cuda_ok(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev)) && coop &&
         cuda_ok(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev))) {
@@ -583,6 +610,10 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
   p.k = c->cfg.kg; p.L = c->geo.L; p.bits = c->geo.gbits;
   p.alpha = alpha;
   p.h = c->h;
+  p.x = c->buf.x;
+  p.wcodes = static_cast<const unsigned char*>(c->buf.wcodes);
+  p.kx = c->cfg.kx; p.xbits = c->geo.xbits;
+  p.lambda = c->lambda;
 
   if (c->geo.gmode == G_IDENTITY) {
     const int grid = (int)std::min<int64_t>(c->grid_ident, p.total_tiles);
@@ -592,7 +623,8 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
     }
     if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
     c->launches += 1;
-  } else if (c->grid_fused > 0 && worker_begin == 0 && worker_count == c->cfg.n) {
+  } else if (c->grid_fused > 0 && worker_begin == 0 && worker_count == c->cfg.n && c->lambda == 0.0f) {
+    // (the pipelined kernel does not stage the held weights: with an l2 term the split kernels run)
     const size_t pairs = (size_t)c->cfg.n * p.S;
     if (!cuda_ok(cudaMemsetAsync(p.scale_bits, 0, sizeof(unsigned) * pairs, c->stream)) ||
         !cuda_ok(cudaMemsetAsync(c->d_done, 0, sizeof(unsigned) * pairs, c->stream)))
@@ -634,6 +666,25 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
     c->launches += 2;
   }
   c->workers_done += worker_count;
+  return QADAM_OK;
+}
+
+int qadam_set_moment_rates(qadam_ctx* c, float beta_t, float theta_t) {
+  if (!c) return QADAM_ERR_NULL;
+  if (!(beta_t >= 0.0f && beta_t < 1.0f) || !(theta_t >= 0.0f && theta_t < 1.0f)) return QADAM_ERR_HYPER;
+  c->h.beta = beta_t;
+  c->h.theta = theta_t;
+  c->h.one_minus_beta = 1.0f - beta_t;
+  c->h.one_minus_theta = 1.0f - theta_t;
+  return QADAM_OK;
+}
+
+int qadam_set_regularization(qadam_ctx* c, float lambda) {
+  if (!c) return QADAM_ERR_NULL;
+  if (!(lambda >= 0.0f) || !std::isfinite(lambda)) return QADAM_ERR_HYPER;
+  const bool changed = (c->lambda != 0.0f) != (lambda != 0.0f);
+  c->lambda = lambda;
+  if (changed) plan_worker_grids(c);
   return QADAM_OK;
 }
 

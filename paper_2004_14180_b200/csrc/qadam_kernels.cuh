@@ -31,7 +31,59 @@ struct WorkerParams {
   int k, L, bits;        // level parameter, positive levels, code width
   float alpha;
   Hyper h;
+  // l2 term (kernels instantiated with L2 = true): lambda * (held weights) is added to g
+  const float* x;               // [D] master copy (held as is when kx < 0)
+  const unsigned char* wcodes;  // packed Q_x(x) (kx >= 0)
+  int kx, xbits;
+  float lambda;
 };
+
+// The weights a worker holds for this lane's 4 elements of a 128-element row: the broadcast
+// Q_x(x) decoded from its packed codes (code - 2^kx times the grid step, exact), or x itself
+// when the weights are not quantized.  row_elem: first element of the row.
+__device__ __forceinline__ void held_weights4(const WorkerParams& p, long long row_elem, int lane,
+                                              float out[4]) {
+  if (p.kx < 0) {
+    const float4 v = *reinterpret_cast<const float4*>(p.x + row_elem + lane * 4);
+    out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
+    return;
+  }
+  const unsigned char* row = p.wcodes + row_elem * p.xbits / 8;
+  const unsigned mask = (1u << p.xbits) - 1u;
+  const float step = exp2i(-(p.kx + 1));
+  // code -> float without a conversion: 2^23 + code as a bit pattern, minus 2^23 + 2^kx
+  const float bias = -(8388608.0f + (float)(1 << p.kx));
+  auto value = [&](unsigned code) {
+    return __fmul_rn(__fadd_rn(__uint_as_float(0x4b000000u | code), bias), step);
+  };
+  if (p.xbits <= 8) {
+    const unsigned f = unpack_row_field(row, p.xbits, lane);          // the lane's 4 codes
+#pragma unroll
+    for (int c = 0; c < 4; ++c) out[c] = value((f >> (c * p.xbits)) & mask);
+    return;
+  }
+  const unsigned* words = reinterpret_cast<const unsigned*>(row);
+  const int row_words = 4 * p.xbits;                    // 128 codes
+  const int half = 2 * p.xbits;                         // two codes, at most 32 bits
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const int bit = 2 * half * lane + h * half;
+    const int w = bit >> 5;
+    const unsigned lo = __ldg(words + w);
+    const unsigned hi = __ldg(words + (w + 1 < row_words ? w + 1 : w));
+    const unsigned f = __funnelshift_r(lo, hi, bit & 31);
+    out[2 * h] = value(f & mask);
+    out[2 * h + 1] = value((f >> p.xbits) & mask);
+  }
+}
+// g + lambda * (held weights), each operation rounded once (Section 5.1's l2 term)
+__device__ __forceinline__ void add_l2_term(const WorkerParams& p, long long row_elem, int lane,
+                                            float gg[4]) {
+  float w[4];
+  held_weights4(p, row_elem, lane, w);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) gg[c] = __fadd_rn(gg[c], __fmul_rn(p.lambda, w[c]));
+}
 
 struct ServerParams {
   float* x;              // [D]
@@ -88,8 +140,8 @@ __device__ __forceinline__ unsigned block_max(unsigned v, unsigned* smem8) {
 // patterns of |u| (monotone for non-negative floats, exact, order-free; a NaN
 // or Inf ends up as the maximum and is reported by phase 2).
 // ---------------------------------------------------------------------------
-template <bool WORKER_MOMENTS>
-__global__ void __launch_bounds__(kThreads)
+template <bool WORKER_MOMENTS, bool L2 = false>
+__global__ void __launch_bounds__(kThreads, WORKER_MOMENTS ? 2 : 4)
 worker_absmax_kernel(const WorkerParams p) {
   __shared__ unsigned red[kThreads / 32];
   unsigned mx = 0;
@@ -131,6 +183,8 @@ worker_absmax_kernel(const WorkerParams p) {
       float gg[4] = {gv[r].x, gv[r].y, gv[r].z, gv[r].w};
       float ee[4] = {ev[r].x, ev[r].y, ev[r].z, ev[r].w};
       float uu[4];
+      if constexpr (L2)
+        add_l2_term(p, tile.off + r * kRowElems + (threadIdx.x >> 5) * 128, threadIdx.x & 31, gg);
       if constexpr (WORKER_MOMENTS) {
         float mm[4] = {mv[r].x, mv[r].y, mv[r].z, mv[r].w};
         float vs[4] = {vv[r].x, vv[r].y, vv[r].z, vv[r].w};
@@ -160,7 +214,7 @@ worker_absmax_kernel(const WorkerParams p) {
 // Worker phase 2: codes = Q_g level indices of u against the finished scale,
 // packed; e <- u - Q_g(u).  U_IN_E: u was left in e's slot by phase 1.
 // ---------------------------------------------------------------------------
-template <bool U_IN_E, int MODE>
+template <bool U_IN_E, int MODE, bool L2 = false>
 __global__ void __launch_bounds__(kThreads)
 worker_quantize_kernel(const WorkerParams p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -196,6 +250,7 @@ worker_quantize_kernel(const WorkerParams p) {
         for (int c = 0; c < 4; ++c) uu[c] = ee[c];
       } else {
         float gg[4] = {gv[r].x, gv[r].y, gv[r].z, gv[r].w};
+        if constexpr (L2) add_l2_term(p, tile.off + r * kRowElems + warp * 128, lane, gg);
 #pragma unroll
         for (int c = 0; c < 4; ++c) uu[c] = __fadd_rn(gg[c], ee[c]);
       }
@@ -220,7 +275,7 @@ worker_quantize_kernel(const WorkerParams p) {
 // ---------------------------------------------------------------------------
 // Identity Q_g: the stream is u itself, the scale is 1, e <- u - u.
 // ---------------------------------------------------------------------------
-template <bool WORKER_MOMENTS>
+template <bool WORKER_MOMENTS, bool L2 = false>
 __global__ void __launch_bounds__(kThreads)
 worker_identity_kernel(const WorkerParams p) {
   for (long long t = blockIdx.x; t < p.total_tiles; t += gridDim.x) {
@@ -244,6 +299,8 @@ worker_identity_kernel(const WorkerParams p) {
       float gg[4] = {g4.x, g4.y, g4.z, g4.w};
       float ee[4] = {e4.x, e4.y, e4.z, e4.w};
       float uu[4], en[4];
+      if constexpr (L2)
+        add_l2_term(p, tile.off + r * kRowElems + (threadIdx.x >> 5) * 128, threadIdx.x & 31, gg);
       if constexpr (WORKER_MOMENTS) {
         const float4 m4 = ld_f4(p.m + so + idx);
         const float4 v4 = ld_f4(p.v + so + idx);

@@ -111,6 +111,7 @@ extern "C" int qadam_worker_scales_static(const float* g, const float* e, int64_
   p.k = 0; p.L = 1; p.bits = 2;
   p.alpha = 0.0f;
   p.h = Hyper{0.0f, 0.0f, 1.0f, 1.0f, 1.0f};
+  p.x = nullptr; p.wcodes = nullptr; p.kx = -1; p.xbits = 0; p.lambda = 0.0f;   // no l2 term
 
   int dev = 0, sms = 0, per_sm = 0;
   if (cudaGetDevice(&dev) != cudaSuccess ||

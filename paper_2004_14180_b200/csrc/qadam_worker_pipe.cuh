@@ -45,6 +45,8 @@ struct __align__(8) Run {
   int seg;
   int phase;              // 0: phase 1, 1: phase 2
   int dir;                // +1: tiles ascending, -1: descending
+  int keep;               // phase 1: ask L2 to hold on to the lines (phase 2 will find them there)
+  int pad;
 };
 
 struct WorkerPipeParams {
@@ -170,12 +172,12 @@ worker_pipe_kernel(const WorkerPipeParams fp, const int stages, const int chunk)
     // header, copy issue, now and then a poll) is paid twice as fast.
     const int pidx = warp - kWConsumers / 32;
     Run* s_run = s_run_all + pidx * kWRunWindow;
-    struct Desc { long long off, pair; int count, phase, worker, need; };
+    struct Desc { long long off, pair; int count, phase, worker, need, keep; };
     int win_base = -1, r = 0;
     // Item t -> its tile.  The run records come through a shared-memory window that
     // the warp refills 128 at a time; runs are ordered by first item, so the run of
     // t is found by bisection from the current one onwards.
-    Run run = Run{0, 0, 0, 0, 0, 0, 0, 1};             // the run of the last item looked up
+    Run run = Run{0, 0, 0, 0, 0, 0, 0, 1, 0, 0};       // the run of the last item looked up
     long long run_end = 0;                             // first item after it (0: none yet)
     auto lookup = [&](long long t) -> Desc {
       while (t >= run_end) {                           // only when the item leaves the current run
@@ -187,7 +189,7 @@ worker_pipe_kernel(const WorkerPipeParams fp, const int stages, const int chunk)
             if (idx < fp.num_runs) {
               s_run[i] = fp.runs[idx];
             } else {
-              Run sentinel = Run{fp.total_items, 0, 0, 0, 0, 0, 0, 1};
+              Run sentinel = Run{fp.total_items, 0, 0, 0, 0, 0, 0, 1, 0, 0};
               s_run[i] = sentinel;
             }
           }
@@ -214,6 +216,7 @@ worker_pipe_kernel(const WorkerPipeParams fp, const int stages, const int chunk)
       d.worker = run.worker;
       d.pair = (long long)run.worker * p.S + run.seg;
       d.need = run.ntiles;
+      d.keep = run.keep;
       return d;
     };
     const unsigned long long keep = policy_evict_last(), drop = policy_evict_first();
@@ -222,7 +225,7 @@ worker_pipe_kernel(const WorkerPipeParams fp, const int stages, const int chunk)
     unsigned armed_mask = 0, armed_par = 0;            // stages this warp has armed, and with which parity
     long long ready_pair = -1;                         // pair whose scale is known to be final
     unsigned ready_scale = 0;
-    Desc cur = Desc{0, 0, 0, 0, 0, 0}, next = cur;
+    Desc cur = Desc{0, 0, 0, 0, 0, 0, 0}, next = cur;
     // item numbers of this CTA, advanced without divisions: `within` counts inside a chunk
     long long t_next = (long long)blockIdx.x * chunk;
     int within = 0;
@@ -251,10 +254,16 @@ worker_pipe_kernel(const WorkerPipeParams fp, const int stages, const int chunk)
         // The copies go out first (g and e are inputs nobody has touched yet); the stage is
         // handed to the consumers by the arrive below, once the header is complete.
         mbar_expect_tx(&ps->full[s], 2u * bytes);
-        const unsigned long long pol = cur.phase == 0 ? keep : drop;
         const long long eo = (long long)cur.worker * p.D + cur.off;
-        bulk_load_hint(st + kWHeaderBytes, p.g + eo, bytes, &ps->full[s], pol);
-        bulk_load_hint(st + kWHeaderBytes + kWTile * 4, p.e + eo, bytes, &ps->full[s], pol);
+        if (cur.phase == 0 && !cur.keep) {
+          // phase 1 of a pair too large for L2: plain streaming loads
+          bulk_load(st + kWHeaderBytes, p.g + eo, bytes, &ps->full[s]);
+          bulk_load(st + kWHeaderBytes + kWTile * 4, p.e + eo, bytes, &ps->full[s]);
+        } else {
+          const unsigned long long pol = cur.phase == 0 ? keep : drop;
+          bulk_load_hint(st + kWHeaderBytes, p.g + eo, bytes, &ps->full[s], pol);
+          bulk_load_hint(st + kWHeaderBytes + kWTile * 4, p.e + eo, bytes, &ps->full[s], pol);
+        }
         if (cur.phase != 0 && cur.pair != ready_pair) {
           // phase 2 needs the pair's scale: wait until all its phase-1 tiles are published
           ok = false;

@@ -63,6 +63,14 @@ class Pair:
         self.gpu.server_step(self.step_no, lr)
         self.cpu.server_step(lr)
 
+    def set_moment_rates(self, beta_t: float, theta_t: float):
+        self.gpu.set_moment_rates(beta_t, theta_t)
+        self.cpu.set_moment_rates(beta_t, theta_t)
+
+    def set_regularization(self, weight_decay: float):
+        self.gpu.set_regularization(weight_decay)
+        self.cpu.set_regularization(weight_decay)
+
     # ------------------------------------------------------------------ checks
     def compare_worker_outputs(self):
         g, c = self.gpu, self.cpu

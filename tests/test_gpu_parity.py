@@ -190,6 +190,53 @@ def test_five_level_sparse_and_dense_code_regions(placement):
     p.close()
 
 
+# ---------------------------------------------------------------- l2 term and step-dependent rates
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+@pytest.mark.parametrize("kg,kx", [(0, 0), (1, 1), (0, 6), (2, 2), (0, -1), (-1, 0), (0, 4), (0, 10), (0, 14)])
+def test_l2_term(kg, kx, placement):
+    """Section 5.1's weight decay: g + lambda * (weights the workers hold), for every width of
+    the packed broadcast the workers decode (2, 3, 4, 6, 8, 12, 16 bits) and for unquantized
+    weights, switched on after one plain step and off again at the end."""
+    rng = np.random.default_rng(300 + 10 * kg + kx)
+    seg, n = [3000, 200, 4100, 64], 3
+    d = sum(seg)
+    x1 = (rng.standard_normal(d) * 0.3).astype(np.float32)
+    p = Pair(seg, n, kg, kx, placement, x1=x1)
+    lam = [0.0, 5e-4, 5e-4, 0.1, 0.0]
+    for t in range(5):
+        p.set_regularization(lam[t])
+        p.step(_rand_grads(rng, n, d), split_workers=t == 2)
+        p.compare_state()
+    p.close()
+
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_step_dependent_rates(placement):
+    """Assumption 2: theta_t = 1 - theta/t, alpha_t = alpha/sqrt(t), a decaying beta_t."""
+    rng = np.random.default_rng(41)
+    seg, n = [5000, 130], 4
+    d = sum(seg)
+    p = Pair(seg, n, 0, 0, placement, x1=(rng.standard_normal(d) * 0.1).astype(np.float32))
+    for t in range(1, 7):
+        p.set_moment_rates(float(np.float32(0.9 * 0.8 ** (t - 1))), float(np.float32(1.0 - 0.5 / t)))
+        p.step(_rand_grads(rng, n, d), lr=float(np.float32(1e-3 / np.sqrt(t))))
+        p.compare_state()
+    p.close()
+
+
+def test_setters_reject_bad_values():
+    import paper_2004_14180_b200 as qb
+    q = qb.QAdam([1000], 1, kg=0, kx=0)
+    for bad in [(1.0, 0.5), (-0.1, 0.5), (0.5, 1.0), (0.5, float("nan"))]:
+        with pytest.raises(qb.QAdamError):
+            q.set_moment_rates(*bad)
+    for bad in [-1e-3, float("inf"), float("nan")]:
+        with pytest.raises(qb.QAdamError):
+            q.set_regularization(bad)
+    q.close()
+
+
 def test_nonfinite_input_sets_status_bit():
     import paper_2004_14180_b200 as qb
     q = qb.QAdam([1000], 1, kg=0, kx=-1)
