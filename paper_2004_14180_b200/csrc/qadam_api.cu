@@ -336,7 +336,9 @@ PipeKernel pick_pipe_n(int n) {
 PipeKernel pick_pipe(const qadam_ctx* c) {
   const bool sm = c->cfg.placement == QADAM_PLACE_SERVER;
   if (c->geo.gmode == G_FIVE) return sm ? pick_pipe_n<true, 3>(c->cfg.n) : pick_pipe_n<false, 3>(c->cfg.n);
-  return sm ? pick_pipe_n<true, 2>(c->cfg.n) : pick_pipe_n<false, 2>(c->cfg.n);
+  if (c->geo.gmode == G_TERNARY) return sm ? pick_pipe_n<true, 2>(c->cfg.n) : pick_pipe_n<false, 2>(c->cfg.n);
+  // any other grid of at most 8 bits: table decode, worker count at run time
+  return sm ? server_pipe_kernel<true, 0, 0> : server_pipe_kernel<false, 0, 0>;
 }
 
 using WorkerPipeKernel = void (*)(const WorkerPipeParams, const int, const int);
@@ -402,6 +404,7 @@ ServerParams make_server_params(const qadam_ctx* c, float alpha) {
   p.S = c->cfg.num_segments;
   p.n = c->cfg.n;
   p.k = c->cfg.kg; p.L = c->geo.L; p.gbits = c->geo.gbits;
+  p.gmode = c->geo.gmode;
   p.kx = c->cfg.kx; p.xbits = c->geo.xbits;
   p.alpha = alpha;
   p.nf = (float)c->cfg.n;
@@ -499,21 +502,23 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
       delete c; return QADAM_ERR_CUDA;
     }
     const bool sm_mom = cfg->placement == QADAM_PLACE_SERVER;
-    const bool pipe_codes = c->geo.gmode == G_TERNARY || c->geo.gmode == G_FIVE;
+    const bool table = c->geo.gmode == G_POW2 || c->geo.gmode == G_UNIFORM;
+    const bool pipe_codes = c->geo.gmode == G_TERNARY || c->geo.gmode == G_FIVE || (table && c->geo.gbits <= 8);
     const size_t sb = pipe_stage_bytes(cfg->n, sm_mom, pipe_codes ? c->geo.gbits : 2);
+    const size_t head = pipe_head_bytes(table);
     const char* env = std::getenv("QADAM_SERVER_KERNEL");
     const bool want_plain = env && std::strcmp(env, "plain") == 0;
-    int stages = (int)(((size_t)max_smem - 256) / sb);
+    int stages = (int)(((size_t)max_smem - head) / sb);
     stages = pipe_legal_stages(std::min(stages, kPipeMaxStages));
     if (!want_plain && pipe_codes && cfg->n <= kPipeMaxWorkers && stages >= 2 &&
         make_codes_tensor_map(&c->codes_map, b->gcodes, (long long)c->geo.gcode_bytes, cfg->n,
-                              c->geo.gbits)) {
+                              c->geo.gbits, table)) {
       c->pipe_stages = stages;
       if (const char* sk16 = std::getenv("QADAM_SKIP_16THS")) {
         const int v = std::atoi(sk16);
         if (v >= 0 && v <= 16) c->pipe_skip_16ths = v;
       }
-      c->pipe_smem = 256 + (size_t)stages * sb;
+      c->pipe_smem = head + (size_t)stages * sb;
       if (!cuda_ok(cudaFuncSetAttribute(pick_pipe(c), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)c->pipe_smem))) {
         delete c; return QADAM_ERR_CUDA;

@@ -100,6 +100,7 @@ struct ServerParams {
   int S;
   int n;
   int k, L, gbits;       // gradient level parameter / levels / code width
+  int gmode;             // GMode of the gradient grid
   int kx, xbits;         // weight level parameter (-1: none) / code width
   float alpha;
   float nf;              // (float)n

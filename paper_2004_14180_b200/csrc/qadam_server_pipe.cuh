@@ -120,8 +120,10 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsig
 // (kPipeTile * gbits / 32) by all n rows: one request brings every worker's codes of a tile, row after row,
 // into shared memory.  Encoded through the driver entry point the runtime hands out,
 // so the library links against the runtime only.  Returns false if unavailable.
+// wide: 64-bit words instead (a box side holds at most 256 elements, which 32-bit words
+// exceed from 5 bits per code on); coordinates and extents are then in 8-byte units.
 inline bool make_codes_tensor_map(CUtensorMap* map, const void* gcodes, long long gcode_bytes, int n,
-                                  int gbits) {
+                                  int gbits, bool wide = false) {
   typedef CUresult (*EncodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -131,12 +133,14 @@ inline bool make_codes_tensor_map(CUtensorMap* map, const void* gcodes, long lon
   if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) != cudaSuccess ||
       qres != cudaDriverEntryPointSuccess || fn == nullptr)
     return false;
-  const cuuint64_t dims[2] = {(cuuint64_t)(gcode_bytes / 4), (cuuint64_t)n};
+  const int word = wide ? 8 : 4;
+  const cuuint64_t dims[2] = {(cuuint64_t)(gcode_bytes / word), (cuuint64_t)n};
   const cuuint64_t strides[1] = {(cuuint64_t)gcode_bytes};          // bytes between rows
-  const cuuint32_t box[2] = {(cuuint32_t)(kPipeTile * gbits / 32), (cuuint32_t)n};
+  const cuuint32_t box[2] = {(cuuint32_t)(kPipeTile * gbits / (8 * word)), (cuuint32_t)n};
+  if (box[0] > 256 || box[1] > 256) return false;
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = reinterpret_cast<EncodeTiled>(fn)(
-      map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(gcodes), dims, strides, box, estr,
+      map, wide ? CU_TENSOR_MAP_DATA_TYPE_UINT64 : CU_TENSOR_MAP_DATA_TYPE_UINT32, 2, const_cast<void*>(gcodes), dims, strides, box, estr,
       CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
       CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
@@ -295,9 +299,15 @@ __device__ __forceinline__ unsigned opaque_u32(unsigned v) {
   return r;
 }
 
+// Bytes ahead of the stage ring: the barriers and, for the table decode, 256 level values.
+__host__ __device__ inline size_t pipe_head_bytes(bool table_decode) {
+  return 256 + (table_decode ? 256 * sizeof(float) : 0);
+}
+
 // NW > 0: the worker count, known at compile time (the decode loop is unrolled and
 // every shared-memory offset is an immediate).  NW = 0: p.n workers, run-time loop.
-// GB: bits per gradient code, 2 (ternary) or 3 (five levels).
+// GB: bits per gradient code, 2 (ternary) or 3 (five levels); 0: any grid with p.gbits
+// (3..8) bits per code, decoded through a table of the signed level values.
 template <bool SERVER_MOMENTS, int NW, int GB>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap codes_map,
@@ -305,18 +315,32 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
                    const int inv_n_exact, const int skip_16ths) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   PipeSmem* ps = reinterpret_cast<PipeSmem*>(smem_raw);
-  unsigned char* stage_base = smem_raw + 256;
+  static_assert(GB == 0 || GB == 2 || GB == 3, "code widths of the pipelined decode");
+  unsigned char* stage_base = smem_raw + pipe_head_bytes(GB == 0);
+  float* s_lut = reinterpret_cast<float*>(smem_raw + 256);      // table decode only
   const int n = NW > 0 ? NW : p.n;
-  static_assert(GB == 2 || GB == 3, "code widths of the pipelined decode");
-  const unsigned stage_bytes = (unsigned)pipe_stage_bytes(n, SERVER_MOMENTS, GB);
+  const int gb = GB > 0 ? GB : p.gbits;
+  const unsigned stage_bytes = (unsigned)pipe_stage_bytes(n, SERVER_MOMENTS, gb);
   constexpr int kState = SERVER_MOMENTS ? 3 : 1;
   constexpr unsigned kCodesOff = kStageHeaderBytes + kState * kPipeTile * 4;
-  constexpr int kRunBytes = kPipeTile * GB / 8;          // one worker's codes of a tile
-  constexpr int kRowBytes = kRunBytes / 2;               // of one of its two 1024-element rows
+  const int kRunBytes = kPipeTile * gb / 8;              // one worker's codes of a tile
+  const int kRowBytes = kRunBytes / 2;                   // of one of its two 1024-element rows
   const unsigned scales_off = kCodesOff + (unsigned)n * kRunBytes;
   const int tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
 
+  if constexpr (GB == 0) {
+    // signed level value of every code (code = level index + L); codes past 2L never occur
+    for (int c = tid; c < 256; c += kPipeThreads) {
+      const int q = c - p.L;
+      const int a = q < 0 ? -q : q;
+      float lv = 0.0f;
+      if (a != 0 && a <= p.L)
+        lv = p.gmode == G_POW2 ? level_value<G_POW2>(a, p.k)
+                               : (p.gmode == G_FIVE ? level_value<G_FIVE>(a, p.k) : level_value<G_UNIFORM>(a, p.k));
+      s_lut[c] = q < 0 ? -lv : lv;
+    }
+  }
   if (tid == 0) {
     for (int s = 0; s < stages; ++s) {
       mbar_init(&ps->full[s], 1);
@@ -386,7 +410,9 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
           bulk_load(sx + kPipeTile, p.m + t.off, fbytes, &ps->full[s]);
           bulk_load(sx + 2 * kPipeTile, p.v + t.off, fbytes, &ps->full[s]);
         }
-        tensor_load_2d(st + kCodesOff, &codes_map, (int)(t.off >> 5) * GB, 0, &ps->full[s]);
+        // coordinate in words of the map: 32-bit (GB > 0) or 64-bit (table decode)
+        const int c0 = GB > 0 ? (int)(t.off >> 5) * GB : (int)(t.off >> 6) * gb;
+        tensor_load_2d(st + kCodesOff, &codes_map, c0, 0, &ps->full[s]);
       }
       ++issued;
       if (++s == stages) { s = 0; ph ^= 1u; }
@@ -449,7 +475,16 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
                             opaque_u32(144u << 23)};
     const FiveLevelLane fl = five_level_lane(lane);          // used by the 3-bit decode only
     // the 3-bit decode holds more per worker in registers: unroll it by 8 at most
-    constexpr int kUnroll = NW > 0 ? (GB == 3 && NW > 8 ? 8 : NW) : 1;
+    constexpr int kUnroll = NW > 0 ? (GB == 0 && NW > 4 ? 4 : (GB == 3 && NW > 8 ? 8 : NW)) : 1;
+    // table decode: the lane's 4 codes are the 4 * gb bits from bit 4 * gb * lane of the
+    // warp's packed row (16 * gb bytes = 4 * gb words)
+    const int tb_word = (4 * gb * lane) >> 5;
+    const int tb_next = tb_word + 1 < 4 * gb ? tb_word + 1 : tb_word;
+    const int tb_shift = (4 * gb * lane) & 31;
+    const unsigned tb_cmask = (1u << gb) - 1u;
+    const unsigned tb_fmask = gb == 8 ? 0xffffffffu : (1u << (4 * gb)) - 1u;
+    unsigned tb_zero = 0;                                    // four level-0 codes
+    for (int c = 0; c < 4; ++c) tb_zero |= (unsigned)p.L << (c * gb);
     bool sparse_mode = true;          // warp-uniform: look for workers with nothing but level 0
     int dense_tiles_left = 0;
     int dense_span = 8;
@@ -464,8 +499,9 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
         if (act0) {
           float* sx = reinterpret_cast<float*>(st + kStageHeaderBytes) + gt * 4;
           // ternary: the thread's byte of a row; five levels: the first of its two bytes
+          // (table decode: the first byte of the warp's packed row)
           const unsigned char* s_codes =
-              st + kCodesOff + (GB == 2 ? gt : gwarp * (128 * GB / 8) + ((lane * 3) >> 1));
+              st + kCodesOff + (GB == 2 ? gt : GB == 3 ? gwarp * 48 + ((lane * 3) >> 1) : gwarp * 16 * gb);
           const bool tiny = GB == 3 && hd.tiny != 0;
           const float2* s_scale = reinterpret_cast<const float2*>(st + scales_off);
           float2 a[4];
@@ -484,12 +520,30 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
             const unsigned char* q = s_codes + i * kRunBytes + r * kRowBytes;
             return (unsigned)q[0] | ((unsigned)q[1] << 8);
           };
+          auto field = [&](int i, int r) -> unsigned {         // table decode: the lane's 4 codes
+            const unsigned* w = reinterpret_cast<const unsigned*>(s_codes + i * kRunBytes + r * kRowBytes);
+            return __funnelshift_r(w[tb_word], w[tb_next], tb_shift);
+          };
+          // value = fl(scale * signed level), then the rounded add: the decode as defined
+          auto table_accumulate = [&](float sc, unsigned f0, unsigned f1) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+              const float v0 = __fmul_rn(sc, s_lut[(f0 >> (c * gb)) & tb_cmask]);
+              const float v1 = __fmul_rn(sc, s_lut[(f1 >> (c * gb)) & tb_cmask]);
+              float2& r0 = a[c >> 1];                          // row 0: a[0], a[1]; row 1: a[2], a[3]
+              float2& r1 = a[2 + (c >> 1)];
+              if (c & 1) { r0.y = __fadd_rn(r0.y, v0); r1.y = __fadd_rn(r1.y, v1); }
+              else       { r0.x = __fadd_rn(r0.x, v0); r1.x = __fadd_rn(r1.x, v1); }
+            }
+          };
           auto contribute = [&](int i) {
             if constexpr (GB == 2) {
               decode_accumulate(s_scale[i], s_codes[i * kRunBytes], s_codes[i * kRunBytes + kRowBytes], k01,
                                 k23, mg, a);
-            } else {
+            } else if constexpr (GB == 3) {
               decode_accumulate5<false>(s_scale[i], window(i, 0), window(i, 1), fl, a);
+            } else {
+              table_accumulate(s_scale[i].x, field(i, 0), field(i, 1));
             }
           };
           auto contribute_pair = [&](int i0, int i1, bool two) {
@@ -500,6 +554,11 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
               const unsigned q0 = s_codes[i1 * kRunBytes], q1 = s_codes[i1 * kRunBytes + kRowBytes];
               decode_accumulate(sc0, p0, p1, k01, k23, mg, a);
               decode_accumulate(sc1, q0, q1, k01, k23, mg, a);
+            } else if constexpr (GB == 0) {
+              const unsigned p0 = field(i0, 0), p1 = field(i0, 1);
+              const unsigned q0 = field(i1, 0), q1 = field(i1, 1);
+              table_accumulate(sc0.x, p0, p1);
+              table_accumulate(sc1.x, q0, q1);
             } else {
               const unsigned p0 = window(i0, 0), p1 = window(i0, 1);
               const unsigned q0 = window(i1, 0), q1 = window(i1, 1);
@@ -513,6 +572,8 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
               const unsigned b0 = s_codes[i * kRunBytes];
               const unsigned b1 = s_codes[i * kRunBytes + kRowBytes];
               nz = (b0 & b1 & 0x55u) != 0x55u;
+            } else if constexpr (GB == 0) {
+              nz = (((field(i, 0) ^ tb_zero) | (field(i, 1) ^ tb_zero)) & tb_fmask) != 0u;
             } else {
               nz = (((window(i, 0) ^ fl.zero) | (window(i, 1) ^ fl.zero)) & fl.field) != 0u;
             }

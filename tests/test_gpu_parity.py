@@ -190,6 +190,32 @@ def test_five_level_sparse_and_dense_code_regions(placement):
     p.close()
 
 
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+@pytest.mark.parametrize("kg,grid", [(2, 0), (2, 1), (3, 1), (6, 1), (14, 0)])
+@pytest.mark.parametrize("n", [1, 16, 33])
+def test_table_decoded_grids(kg, grid, n, placement):
+    """Grids beyond five levels go through the server pipeline's table decode: 3, 4, 5, 8 and
+    5 bits per code here, fields that straddle 32-bit words, several tiles and a ragged tail."""
+    _run([3 * 2048 + 640, 130, 4096], n, kg, 1, placement, T=2, grid=grid, seed=500 + 7 * kg + grid + n)
+
+
+def test_table_decoded_grid_sparse_and_dense_regions():
+    rng = np.random.default_rng(79)
+    d, n = 1 << 22, 8
+    dense_end = d * 3 // 10
+    p = Pair([d], n, 3, 0, S_MODE, x1=(rng.standard_normal(d) * 0.05).astype(np.float32))
+    for t in range(2):
+        g = (rng.standard_normal((n, d)) * 1e-5).astype(np.float32)
+        g[:, :dense_end] = rng.standard_normal((n, dense_end)).astype(np.float32)
+        hits = rng.integers(dense_end, d, (n, 300))
+        for i in range(n):
+            g[i, hits[i]] = rng.choice(np.array([4.0, -4.0, 1.0, -0.5], np.float32), 300)
+        g[:, d - 1] = 5.0
+        p.step(g, threads=4)
+    p.compare_state()
+    p.close()
+
+
 # ---------------------------------------------------------------- l2 term and step-dependent rates
 
 @pytest.mark.parametrize("placement", [S_MODE, W_MODE])
