@@ -153,7 +153,7 @@ class ClockSampler:
 # ----------------------------------------------------------------------------- byte accounting
 
 def algorithmic_bytes(kernel: str, w, placement: str, D: int, gbits: int, xbits: int,
-                      pass_model=None, l2_term: bool = False) -> float:
+                      pass_model=None, l2_term: bool = False, fused_covers_all=None) -> float:
     """Bytes one launch of `kernel` must move at its interface (fp32 state it has
     to read and write, packed codes), for all n workers.  For the fused worker kernel
     the figure is capacity aware: (worker, segment) pairs that fit the kernel's L2
@@ -165,16 +165,20 @@ def algorithmic_bytes(kernel: str, w, placement: str, D: int, gbits: int, xbits:
     held = ((xbits / 8.0) if xbits else 4.0) if l2_term else 0.0
     if kernel == "worker_fused":
         one_pass, two_pass = pass_model
+        if fused_covers_all is False:   # the on-chip kernel: one-pass pairs only
+            return one_pass * (12.0 + gbits / 8.0)
         if server_moments:      # read g, e (twice when two-pass); write e and the codes
             return one_pass * (12.0 + gbits / 8.0) + two_pass * (20.0 + gbits / 8.0)
         # read g, m, v, e; write m, v, e and codes; two-pass adds a write and a read of u
         return one_pass * (28.0 + gbits / 8.0) + two_pass * (36.0 + gbits / 8.0)
+    # the split launches cover everything, or, beside the fused kernel, the two-pass pairs only
+    split_units = pass_model[1] if pass_model and pass_model[0] > 0 else n * D
     if kernel == "absmax":      # phase 1: read g, e (worker moments: + read m, v, write m, v, u)
         per = (8.0 if server_moments else 28.0) + held
-        return per * n * D
+        return per * split_units
     if kernel == "quantize":    # phase 2: read g, e (or u), write e and the codes
         per = (12.0 + held if server_moments else 8.0) + gbits / 8.0
-        return per * n * D
+        return per * split_units
     if kernel == "identity":
         per = ((8.0 + 8.0) if server_moments else (16.0 + 16.0)) + held
         return per * n * D
@@ -378,7 +382,9 @@ def run_b200(args):
             continue
         per = ms / cnt
         bytes_ = algorithmic_bytes(name, w, args.placement, D, q.gcode_bytes * 8 // D, q.wcode_bytes * 8 // D,
-                                   pass_model=q.worker_pass_model(), l2_term=args.weight_decay != 0.0)
+                                   pass_model=q.worker_pass_model(), l2_term=args.weight_decay != 0.0,
+                                   fused_covers_all=not ("absmax" in prof and prof["absmax"][1] > 0
+                                                         and "worker_fused" in prof and prof["worker_fused"][1] > 0))
         kernels[name] = {"launches": int(cnt), "ms_per_launch": per,
                          "share": ms / sum(m for m, c in prof.values()),
                          "algorithmic_bytes": bytes_, "achieved_gbs": bytes_ / (per * 1e-3) / 1e9,

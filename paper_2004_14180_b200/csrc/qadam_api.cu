@@ -14,6 +14,7 @@
 #include "qadam_kernels.cuh"
 #include "qadam_server_pipe.cuh"
 #include "qadam_worker_pipe.cuh"
+#include "qadam_worker_resident.cuh"
 
 #include <cstdlib>
 
@@ -64,7 +65,31 @@ struct Geometry {
   long long one_pass_elems = 0;      // padded (worker, element) pairs in groups that fit the L2 budget
   long long two_pass_elems = 0;      // ... in pairs larger than a group
   size_t off_ptiles = 0, off_runs = 0, off_done = 0;
+  // on-chip worker kernel: tiles of the segments that fit on chip (one vector) and the tiles
+  // of the remaining segments (two streaming passes)
+  std::vector<RTile> rtiles;
+  std::vector<Tile> btiles;
+  long long resident_elems = 0;      // padded elements of the resident segments (one vector)
+  size_t off_rtiles = 0, off_btiles = 0;
 };
+
+// Splits the segments into those the on-chip worker kernel can hold (at most `capacity`
+// tiles per (worker, segment) pair) and the rest, each with a tile table of its own.
+void build_resident(long long capacity, Geometry* g) {
+  g->rtiles.clear();
+  g->btiles.clear();
+  g->resident_elems = 0;
+  for (const Tile& t : g->tiles) {
+    if (g->seg_tiles[t.seg] <= capacity) {
+      RTile r;
+      r.off = t.off; r.count = t.count; r.seg = t.seg; r.need = g->seg_tiles[t.seg]; r.pad = 0;
+      g->rtiles.push_back(r);
+      g->resident_elems += t.count;
+    } else {
+      g->btiles.push_back(t);
+    }
+  }
+}
 
 // Bytes of g + e (server moments) or g, m, v, e + the u written back (worker moments)
 // that one group of (worker, segment) pairs may hold: a few groups must fit in L2
@@ -225,6 +250,11 @@ int build_geometry(const qadam_config* c, Geometry* g) {
   wo += (size_t)round_up64((int64_t)g->runs.size() * sizeof(Run), 256);
   g->off_done = wo;
   wo += (size_t)round_up64((int64_t)c->n * c->num_segments * sizeof(unsigned), 256);
+  // upper bounds (the split into resident and other segments is made at creation, on the device's sizes)
+  g->off_rtiles = wo;
+  wo += (size_t)round_up64((int64_t)g->tiles.size() * sizeof(RTile), 256);
+  g->off_btiles = wo;
+  wo += (size_t)round_up64((int64_t)g->tiles.size() * sizeof(Tile), 256);
   g->workspace_bytes = wo + 256;
   return QADAM_OK;
 }
@@ -258,6 +288,12 @@ struct qadam_ctx {
   size_t wpipe_smem = 0;
   Run* d_runs = nullptr;
   unsigned* d_done = nullptr;
+  // on-chip worker kernel (moments on the server, all workers in one call): grid > 0 when in use
+  int grid_resident = 0;
+  int res_slots = 0, res_estages = 0;
+  size_t res_smem = 0;
+  RTile* d_rtiles = nullptr;
+  Tile* d_btiles = nullptr;
   // instrumentation: event pairs of the launches since the last read
   bool profiling = false;
   struct Timed { int kind; cudaEvent_t start, stop; };
@@ -349,6 +385,17 @@ WorkerPipeKernel pick_worker_pipe(const qadam_ctx* c) {
     case G_FIVE:    return worker_pipe_kernel<G_FIVE>;
     case G_POW2:    return worker_pipe_kernel<G_POW2>;
     default:        return worker_pipe_kernel<G_UNIFORM>;
+  }
+}
+
+using WorkerResidentKernel = void (*)(const WorkerResidentParams);
+
+WorkerResidentKernel pick_worker_resident(const qadam_ctx* c) {
+  switch (c->geo.gmode) {
+    case G_TERNARY: return worker_resident_kernel<G_TERNARY>;
+    case G_FIVE:    return worker_resident_kernel<G_FIVE>;
+    case G_POW2:    return worker_resident_kernel<G_POW2>;
+    default:        return worker_resident_kernel<G_UNIFORM>;
   }
 }
 
@@ -478,6 +525,8 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
     c->d_ptiles = reinterpret_cast<Tile*>(ws + c->geo.off_ptiles);
     c->d_runs = reinterpret_cast<Run*>(ws + c->geo.off_runs);
     c->d_done = reinterpret_cast<unsigned*>(ws + c->geo.off_done);
+    c->d_rtiles = reinterpret_cast<RTile*>(ws + c->geo.off_rtiles);
+    c->d_btiles = reinterpret_cast<Tile*>(ws + c->geo.off_btiles);
   }
 
   int dev = 0;
@@ -528,19 +577,23 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
   plan_worker_grids(c);
   c->grid_server = resident_grid(sk, c->server_smem, c->sm_count);
   c->grid_bcast = resident_grid(weight_broadcast_kernel, 0, c->sm_count);
-  // The pipelined worker kernel needs every CTA resident at once (its phase-2 items wait
-  // for phase-1 items of other CTAs): one CTA per SM, launched cooperatively.  It pays
-  // through the (worker, segment) pairs that stay in L2 between the phases; when no pair
-  // does (every segment larger than a group) the two plain streaming launches are a few
-  // per cent faster (measured) and run instead, unless QADAM_WORKER_KERNEL=pipe.
+  // Worker side, moments on the server, all workers in one call.  Segments small enough
+  // for a wave of the on-chip kernel (u = g + e stays in shared memory between the
+  // max-abs reduction and the quantization, so g and e are read once) go through that
+  // kernel; larger segments need two passes over memory whatever is done and take the two
+  // plain streaming launches, over a tile table of their own.  The on-chip kernel needs
+  // every CTA resident at once (its store side waits for other CTAs' load sides): one
+  // CTA per SM, launched cooperatively.
+  // QADAM_WORKER_KERNEL=split: streaming launches only; =pipe: the L2-group pipeline.
   {
     int coop = 0, max_smem = 0;
     const char* env = std::getenv("QADAM_WORKER_KERNEL");
-    const bool want_split = (env && std::strcmp(env, "split") == 0) ||
-                            (c->geo.one_pass_elems == 0 && !(env && std::strcmp(env, "pipe") == 0));
-    if (!want_split && c->geo.gmode != G_IDENTITY && cfg->placement == QADAM_PLACE_SERVER &&
+    const bool want_split = env && std::strcmp(env, "split") == 0;
+    const bool want_pipe = env && std::strcmp(env, "pipe") == 0;
+    const bool eligible = !want_split && c->geo.gmode != G_IDENTITY && cfg->placement == QADAM_PLACE_SERVER &&
         cuda_ok(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev)) && coop &&
-        cuda_ok(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev))) {
+        cuda_ok(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    if (eligible && want_pipe) {
       int stages = (int)(((size_t)max_smem - wpipe_smem_bytes(0)) / kWStageBytes);
       stages = std::min(stages, kWMaxStages) / kWGroups * kWGroups;
       if (stages >= kWGroups) {
@@ -557,6 +610,30 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
             per_sm >= 1)
           c->grid_fused = c->sm_count;
       }
+    } else if (eligible) {
+      // the CTA's shared memory: a ring of slots for u and a few stages for e (227 KB: 14 in all)
+      const char* ee = std::getenv("QADAM_RESIDENT_ESTAGES");
+      int estages = ee ? std::atoi(ee) : 3;
+      estages = std::max(2, std::min(estages, kRMaxEStages));
+      const int slots = std::min(((int)max_smem - kRHeadBytes) / kRSlotBytes - estages, kRMaxSlots);
+      // a pair may give a CTA at most slots - 2 tiles: the rest of the ring lets the load side
+      // run ahead into the next pair while this one is quantized and stored
+      const char* me = std::getenv("QADAM_RESIDENT_SPARE");
+      const int spare = std::max(1, me ? std::atoi(me) : 2);
+      if (slots - spare >= 1) {
+        build_resident((long long)c->sm_count * (slots - spare), &c->geo);
+        c->res_slots = slots;
+        c->res_estages = estages;
+        c->res_smem = resident_smem_bytes(slots, estages);
+        int per_sm = 0;
+        if (!c->geo.rtiles.empty() &&
+            cuda_ok(cudaFuncSetAttribute(pick_worker_resident(c), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)c->res_smem)) &&
+            cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pick_worker_resident(c), kRThreads,
+                                                                  c->res_smem)) &&
+            per_sm >= 1)
+          c->grid_resident = c->sm_count;
+      }
     }
   }
   if (c->grid_absmax < 0 || c->grid_quant < 0 || c->grid_ident < 0 || c->grid_server < 0 ||
@@ -571,6 +648,12 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
                                cudaMemcpyHostToDevice, c->stream)) ||
       !cuda_ok(cudaMemcpyAsync(c->d_runs, c->geo.runs.data(), c->geo.runs.size() * sizeof(Run),
                                cudaMemcpyHostToDevice, c->stream)) ||
+      (c->grid_resident > 0 &&
+       (!cuda_ok(cudaMemcpyAsync(c->d_rtiles, c->geo.rtiles.data(), c->geo.rtiles.size() * sizeof(RTile),
+                                 cudaMemcpyHostToDevice, c->stream)) ||
+        (!c->geo.btiles.empty() &&
+         !cuda_ok(cudaMemcpyAsync(c->d_btiles, c->geo.btiles.data(), c->geo.btiles.size() * sizeof(Tile),
+                                  cudaMemcpyHostToDevice, c->stream))))) ||
       !cuda_ok(cudaMemsetAsync(b->status, 0, sizeof(uint32_t), c->stream)) ||
       !cuda_ok(cudaStreamSynchronize(c->stream))) {
     delete c; return QADAM_ERR_CUDA;
@@ -628,6 +711,48 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
     }
     if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
     c->launches += 1;
+  } else if (c->grid_resident > 0 && worker_begin == 0 && worker_count == c->cfg.n && c->lambda == 0.0f) {
+    // (the on-chip kernel does not stage the held weights: with an l2 term the split kernels run)
+    const size_t pairs = (size_t)c->cfg.n * p.S;
+    if (!cuda_ok(cudaMemsetAsync(p.scale_bits, 0, sizeof(unsigned) * pairs, c->stream)) ||
+        !cuda_ok(cudaMemsetAsync(c->d_done, 0, sizeof(unsigned) * pairs, c->stream)))
+      return QADAM_ERR_CUDA;
+    WorkerResidentParams rp;
+    rp.w = p;
+    rp.rtiles = c->d_rtiles;
+    rp.done = c->d_done;
+    rp.TR = (int)c->geo.rtiles.size();
+    rp.total = (long long)c->cfg.n * rp.TR;
+    rp.slots = c->res_slots;
+    rp.estages = c->res_estages;
+    void* args[] = {&rp};
+    cudaError_t e;
+    {
+      LaunchTimer lt(c, QADAM_K_WORKER_FUSED);
+      e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(pick_worker_resident(c)),
+                                      dim3(c->grid_resident), dim3(kRThreads), args, c->res_smem, c->stream);
+    }
+    if (!cuda_ok(e)) return QADAM_ERR_CUDA;
+    c->launches += 1;
+    if (!c->geo.btiles.empty()) {
+      // the segments too large for a wave: two streaming passes over their own tile table
+      p.tiles = c->d_btiles;
+      p.tiles_per_worker = (int)c->geo.btiles.size();
+      p.total_tiles = (long long)worker_count * p.tiles_per_worker;
+      int grid = (int)std::min<int64_t>(c->grid_absmax, p.total_tiles);
+      {
+        LaunchTimer lt(c, QADAM_K_ABSMAX);
+        pick_absmax(c)<<<grid, kThreads, 0, c->stream>>>(p);
+      }
+      if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
+      grid = (int)std::min<int64_t>(c->grid_quant, p.total_tiles);
+      {
+        LaunchTimer lt(c, QADAM_K_QUANTIZE);
+        pick_quantize(c)<<<grid, kThreads, 0, c->stream>>>(p);
+      }
+      if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
+      c->launches += 2;
+    }
   } else if (c->grid_fused > 0 && worker_begin == 0 && worker_count == c->cfg.n && c->lambda == 0.0f) {
     // (the pipelined kernel does not stage the held weights: with an l2 term the split kernels run)
     const size_t pairs = (size_t)c->cfg.n * p.S;
@@ -776,7 +901,13 @@ int qadam_profile_read(qadam_ctx* c, double* ms, int64_t* launches) {
 
 int qadam_worker_pass_model(const qadam_ctx* c, int64_t* one_pass, int64_t* two_pass) {
   if (!c || !one_pass || !two_pass) return QADAM_ERR_NULL;
-  if (c->grid_fused > 0) {
+  if (c->lambda != 0.0f) {              // with the l2 term the split launches cover everything
+    *one_pass = 0;
+    *two_pass = (int64_t)c->cfg.n * c->geo.D;
+  } else if (c->grid_resident > 0) {
+    *one_pass = (int64_t)c->cfg.n * c->geo.resident_elems;
+    *two_pass = (int64_t)c->cfg.n * (c->geo.D - c->geo.resident_elems);
+  } else if (c->grid_fused > 0) {
     *one_pass = c->geo.one_pass_elems;
     *two_pass = c->geo.two_pass_elems;
   } else {

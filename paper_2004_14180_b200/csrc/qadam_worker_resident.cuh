@@ -1,0 +1,386 @@
+// The worker side (moments on the server) for tensors that fit ON CHIP: one persistent
+// kernel that reads g and e once, keeps u = g + e in shared memory until the tensor's
+// scale is known, and quantizes from there.
+//
+// The scale of Q_g is the maximum of |u| over a whole (worker, segment) pair, so no
+// element of a pair can be quantized before all of the pair has been read.  Going back
+// to memory for the second look costs as much through L2 as from HBM on this machine
+// (the path from L2 into an SM carries little more than HBM delivers: measured), so the
+// only way to touch each element once is to hold u where it was computed.  Each of the
+// 148 SMs keeps a ring of 10 to 12 slots of 4096 values; a pair spread over all SMs may
+// therefore be up to a few million elements long.  Per pair and element this moves g, e
+// in and e', the packed code out: 12 + b_g / 8 bytes, the least the method allows.
+//
+// The resident tiles of all workers are numbered worker-major, t = worker * TR + j
+// (j: index in the per-vector list of resident tiles), so the tiles of a pair are
+// consecutive.  Tile t belongs to CTA t mod gridDim.x; a CTA takes its tiles in
+// increasing order and its i-th tile lives in slot i mod slots.  Per CTA, one per SM:
+//   load side    a producer warp brings g into the tile's slot and e into a small ring
+//                with bulk copies that complete on an mbarrier; eight consumer warps
+//                add e to g in place and fold max |u|; a publisher warp adds the CTA's
+//                maximum and tile count to the pair's global record;
+//   store side   a dispatcher warp waits until all tiles of the pair have been counted
+//                (every CTA's, hence the final scale), sixteen consumer warps quantize the
+//                slot, write the packed codes and leave e' in the slot; a storer warp
+//                sends e' back with a bulk store and frees the slot.
+// The two sides run as independent loops over the CTA's tiles, coupled only by the
+// pair records in global memory and the slots' "free" barriers: the load side runs
+// ahead of the store side by as many tiles as there are slots, which is what hides the
+// latency of the grid-wide hand-over (last load of a pair lands somewhere -> every CTA
+// learns the scale).  No deadlock: a load waits for the store of the tile `slots`
+// places earlier in the same CTA, which waits for that tile's pair to be complete, which
+// waits for loads of that pair only; a pair gives a CTA fewer tiles than it has slots
+// (the host sends larger pairs elsewhere), so those loads wait, in turn, only for
+// stores of OLDER pairs, and the oldest unfinished pair can always finish, provided
+// every CTA is resident (cooperative launch).  All waits are bounded: when one runs out
+// the TIMEOUT bit of the status word is set and every role leaves its loop.
+#pragma once
+
+#include "qadam_worker_pipe.cuh"
+
+namespace qadam {
+
+// A tile of a resident segment (padded layout, one vector).
+struct __align__(8) RTile {
+  long long off;   // first element
+  int count;       // elements, multiple of kAlign, at most kTileElems
+  int seg;         // segment
+  int need;        // tiles of that segment: what the pair's counter must reach
+  int pad;
+};
+
+struct WorkerResidentParams {
+  WorkerParams w;
+  const RTile* rtiles;    // [TR]
+  unsigned* done;         // [n][S] tiles counted per pair, zeroed before the launch (as are the scales)
+  long long total;        // n * TR resident tiles in all
+  int TR;                 // resident tiles per worker
+  int slots;              // slots of the CTA's ring (a pair gives a CTA fewer tiles than this)
+  int estages;            // stages of the e ring
+};
+
+#ifndef QADAM_RESIDENT_QWARPS
+#define QADAM_RESIDENT_QWARPS 16
+#endif
+constexpr int kRGroupThreads = 256;     // load-side consumers: 8 warps, 4 rows of 1024 elements per tile
+constexpr int kRQWarps = QADAM_RESIDENT_QWARPS;   // store-side consumers: 8 or 16 warps (4 or 2 rows per thread)
+constexpr int kRQRowStep = kRQWarps / 8;
+constexpr int kRRoleWarp0 = 8 + kRQWarps;         // producer, publisher, dispatcher, storer follow
+constexpr int kRThreads = 32 * (kRRoleWarp0 + 4);
+static_assert(kRQWarps == 8 || kRQWarps == 16, "store-side consumer warps");
+constexpr int kRSlotBytes = kTileElems * 4;
+constexpr int kRCmds = 4;               // quantize commands in flight
+constexpr int kRMaxEStages = 8;
+constexpr int kRMaxSlots = 16;
+constexpr int kRHeaders = 32;           // ring of tile headers; more than slots + e stages, see the publisher
+constexpr int kRHeadBytes = 2048;       // barriers, headers, commands
+
+struct RLoadHeader {       // one per tile in flight on the load side (ring of kRHeaders)
+  long long pair;          // worker * S + segment
+  int slot;                // where g lands and u stays
+  int count;               // elements of the tile
+  int publish;             // last tile of the CTA's streak of this pair
+  unsigned max_bits;       // max |u| of the tile, folded in by the consumer warps
+};
+struct RCommand {          // one per quantize command
+  long long off;           // first element (padded layout)
+  int slot;
+  int count;
+  int worker;
+  unsigned scale_bits;     // the pair's final scale
+};
+
+struct RSmem {
+  unsigned long long e_full[kRMaxEStages];
+  unsigned long long e_empty[kRMaxEStages];
+  unsigned long long hd_ready[kRHeaders];     // consumers -> publisher: the tile's maximum is in its header
+  unsigned long long slot_free[kRMaxSlots];
+  unsigned long long cmd_full[kRCmds];
+  unsigned long long cmd_computed[kRCmds];
+  unsigned long long cmd_empty[kRCmds];
+  RLoadHeader load_hd[kRHeaders];
+  RCommand cmd[kRCmds];
+  int abort_flag;
+};
+static_assert(sizeof(RSmem) <= kRHeadBytes, "head of the shared-memory layout");
+
+__host__ __device__ inline size_t resident_smem_bytes(int slots, int estages) {
+  return kRHeadBytes + (size_t)(slots + estages) * kRSlotBytes;
+}
+
+template <int MODE>
+__global__ void __launch_bounds__(kRThreads, 1)
+worker_resident_kernel(const WorkerResidentParams rp) {
+  extern __shared__ __align__(128) unsigned char smem_raw[];
+  RSmem* ps = reinterpret_cast<RSmem*>(smem_raw);
+  unsigned char* slot_base = smem_raw + kRHeadBytes;
+  unsigned char* ering_base = slot_base + (size_t)rp.slots * kRSlotBytes;
+  const WorkerParams& p = rp.w;
+  const int tid = threadIdx.x;
+  const int warp = tid >> 5, lane = tid & 31;
+  const int cta = (int)blockIdx.x, ctas = (int)gridDim.x;
+  const int estages = rp.estages;
+
+  if (tid == 0) {
+    for (int s = 0; s < estages; ++s) {
+      mbar_init(&ps->e_full[s], 1);
+      mbar_init(&ps->e_empty[s], kRGroupThreads / 32);
+    }
+    for (int s = 0; s < kRHeaders; ++s) mbar_init(&ps->hd_ready[s], kRGroupThreads / 32);
+    for (int s = 0; s < rp.slots; ++s) mbar_init(&ps->slot_free[s], 1);
+    for (int s = 0; s < kRCmds; ++s) {
+      mbar_init(&ps->cmd_full[s], 1);
+      mbar_init(&ps->cmd_computed[s], kRQWarps);
+      mbar_init(&ps->cmd_empty[s], 1);
+    }
+    ps->abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+  volatile int* abort_flag = &ps->abort_flag;
+  // the CTA's tiles: t = cta, cta + ctas, ... < total
+  const long long my_tiles = cta < rp.total ? (rp.total - cta + ctas - 1) / ctas : 0;
+
+  if (warp == kRRoleWarp0) {
+    // ------------------------------------------------------------------ load side: producer
+    int s = 0;
+    unsigned ph = 0;
+    int slot = 0;
+    unsigned slot_ph = 0;                  // parity of the number of times the ring of slots has been gone round
+    unsigned armed_mask = 0, armed_par = 0;
+    bool ok = true;
+    long long t = cta;
+    int worker = my_tiles > 0 ? (int)(t / rp.TR) : 0;
+    int j = my_tiles > 0 ? (int)(t - (long long)worker * rp.TR) : 0;
+    RTile cur = my_tiles > 0 ? rp.rtiles[j] : RTile{0, 0, 0, 0, 0};
+    for (long long i = 0; i < my_tiles; ++i, t += ctas) {
+      // the CTA's next tile, for the end of the streak of tiles of one pair
+      int worker_n = worker, jn = j + ctas;
+      while (jn >= rp.TR) { jn -= rp.TR; ++worker_n; }
+      RTile next = cur;
+      const bool has_next = i + 1 < my_tiles;
+      if (has_next) next = rp.rtiles[jn];
+      const int publish = !(has_next && worker_n == worker && next.seg == cur.seg);
+      if (lane == 0) {
+        // the slot must have been read out by the store side (a fresh barrier passes a wait on
+        // the parity opposite to its first phase), the ring stage by the consumers
+        ok = mbar_wait_bounded(&ps->slot_free[slot], slot_ph ^ 1u, abort_flag, p.status) &&
+             mbar_wait_bounded(&ps->e_empty[s], ph ^ 1u, abort_flag, p.status);
+        if (ok) {
+          RLoadHeader* hd = &ps->load_hd[i & (kRHeaders - 1)];
+          hd->pair = (long long)worker * p.S + cur.seg;
+          hd->slot = slot;
+          hd->count = cur.count;
+          hd->publish = publish;
+          hd->max_bits = 0u;
+          const unsigned bytes = (unsigned)cur.count * 4u;
+          const long long eo = (long long)worker * p.D + cur.off;
+          mbar_arrive_expect_tx(&ps->e_full[s], 2u * bytes);
+          bulk_load(slot_base + (size_t)slot * kRSlotBytes, p.g + eo, bytes, &ps->e_full[s]);
+          bulk_load(ering_base + (size_t)s * kRSlotBytes, p.e + eo, bytes, &ps->e_full[s]);
+        }
+      }
+      ok = __shfl_sync(0xffffffffu, ok, 0);
+      if (!ok) break;
+      armed_mask |= 1u << s;
+      armed_par = (armed_par & ~(1u << s)) | (ph << s);
+      if (++s == estages) { s = 0; ph ^= 1u; }
+      if (++slot == rp.slots) { slot = 0; slot_ph ^= 1u; }
+      worker = worker_n;
+      j = jn;
+      cur = next;
+    }
+    // drain after an abort: nothing may still be landing in shared memory when the CTA exits
+    __syncwarp();
+    if (lane == 0 && *abort_flag) {
+      for (int ds = 0; ds < estages; ++ds) {
+        if (!((armed_mask >> ds) & 1u)) continue;
+        for (unsigned it = 0; it < kSpinLimit; ++it) {
+          if (mbar_try_wait(&ps->e_full[ds], (armed_par >> ds) & 1u)) break;
+          __nanosleep(100);
+        }
+      }
+    }
+  } else if (warp == kRRoleWarp0 + 1) {
+    // ------------------------------------------------------------------ load side: publisher
+    // The publisher may fall behind the consumers (its atomics take a round trip to L2), so
+    // it has a barrier and a header per tile in a ring of its own rather than sharing the e
+    // stages.  It cannot fall behind by a whole ring: the producer reuses a slot only after
+    // the tile that held it has been stored, which needs that tile's pair complete, which
+    // needs this warp to have published it, and kRHeaders exceeds the slots.
+    unsigned acc_max = 0, acc_cnt = 0;
+    if (lane == 0) {
+      for (long long i = 0; i < my_tiles; ++i) {
+        const int hi = (int)(i & (kRHeaders - 1));
+        if (!mbar_wait_bounded(&ps->hd_ready[hi], (unsigned)(i / kRHeaders) & 1u, abort_flag, p.status)) break;
+        const RLoadHeader hd = ps->load_hd[hi];
+        acc_max = max(acc_max, hd.max_bits);
+        acc_cnt += 1;
+        if (hd.publish) {
+          // the maximum first, then (fence) the count that lets the store side of this pair go
+          if (acc_max) atomicMax(p.scale_bits + hd.pair, acc_max);
+          __threadfence();
+          atomicAdd(rp.done + hd.pair, acc_cnt);
+          acc_max = 0;
+          acc_cnt = 0;
+        }
+      }
+    }
+  } else if (warp == kRRoleWarp0 + 2) {
+    // ------------------------------------------------------------------ store side: dispatcher
+    int cs = 0;
+    unsigned cph = 0;
+    long long ready_pair = -1;
+    unsigned ready_scale = 0;
+    bool ok = true;
+    if (lane == 0 && my_tiles > 0) {
+      long long t = cta;
+      int worker = (int)(t / rp.TR);
+      int j = (int)(t - (long long)worker * rp.TR);
+      int slot = 0;
+      for (long long i = 0; i < my_tiles; ++i) {
+        const RTile cur = rp.rtiles[j];
+        const long long pair = (long long)worker * p.S + cur.seg;
+        if (pair != ready_pair) {
+          ok = false;
+          for (unsigned it = 0; it < kWSpinLimit; ++it) {
+            if (ld_acquire_u32(rp.done + pair) >= (unsigned)cur.need) { ok = true; break; }
+            if (*abort_flag) break;
+            __nanosleep(it < 64 ? 40 : 400);
+          }
+          if (!ok) {
+            if (!*abort_flag) atomicOr(p.status, 2u);
+            *abort_flag = 1;
+            break;
+          }
+          ready_pair = pair;
+          ready_scale = __ldcg(p.scale_bits + pair);
+          if (ready_scale >= 0x7f800000u) atomicOr(p.status, 1u);
+        }
+        ok = mbar_wait_bounded(&ps->cmd_empty[cs], cph ^ 1u, abort_flag, p.status);
+        if (!ok) break;
+        RCommand* cd = &ps->cmd[cs];
+        cd->off = cur.off;
+        cd->slot = slot;
+        cd->count = cur.count;
+        cd->worker = worker;
+        cd->scale_bits = ready_scale;
+        mbar_arrive(&ps->cmd_full[cs]);
+        if (++cs == kRCmds) { cs = 0; cph ^= 1u; }
+        if (++slot == rp.slots) slot = 0;
+        j += ctas;
+        while (j >= rp.TR) { j -= rp.TR; ++worker; }
+      }
+    }
+  } else if (warp == kRRoleWarp0 + 3) {
+    // ------------------------------------------------------------------ store side: storer
+    int cs = 0;
+    unsigned cph = 0;
+    int owed_slot = -1;                      // slot of the last e' store, not yet freed
+    if (lane == 0) {
+      for (long long i = 0; i < my_tiles; ++i) {
+        if (!mbar_wait_bounded(&ps->cmd_computed[cs], cph, abort_flag, p.status)) break;
+        const RCommand cd = ps->cmd[cs];
+        mbar_arrive(&ps->cmd_empty[cs]);
+        bulk_store(p.e + (long long)cd.worker * p.D + cd.off, slot_base + (size_t)cd.slot * kRSlotBytes,
+                   (unsigned)cd.count * 4u);
+        bulk_commit();
+        if (++cs == kRCmds) { cs = 0; cph ^= 1u; }
+        // A slot is freed once the copy engine has read it.  If the next tile is ready, that
+        // wait is put off by one store so that this warp does not sit in it; if not, there
+        // is nothing better to do than to wait here.
+        const bool next_ready = i + 1 < my_tiles && mbar_try_wait(&ps->cmd_computed[cs], cph);
+        if (next_ready) {
+          if (owed_slot >= 0) {
+            bulk_wait_read_1();
+            mbar_arrive(&ps->slot_free[owed_slot]);
+          }
+          owed_slot = cd.slot;
+        } else {
+          bulk_wait_read_all();
+          if (owed_slot >= 0) mbar_arrive(&ps->slot_free[owed_slot]);
+          mbar_arrive(&ps->slot_free[cd.slot]);
+          owed_slot = -1;
+        }
+      }
+      bulk_wait_all();                       // writes are complete before the kernel ends
+    }
+  } else if (warp < 8) {
+    // ------------------------------------------------------------------ load side: u = g + e, max |u|
+    const int gt = tid;                      // 0..255
+    int s = 0;
+    unsigned ph = 0;
+    for (long long i = 0; i < my_tiles; ++i) {
+      if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->e_full[s], ph, abort_flag, p.status))) break;
+      RLoadHeader* hdp = &ps->load_hd[i & (kRHeaders - 1)];
+      const int slot = hdp->slot, count = hdp->count;
+      float* su = reinterpret_cast<float*>(slot_base + (size_t)slot * kRSlotBytes) + gt * 4;
+      const float* se = reinterpret_cast<const float*>(ering_base + (size_t)s * kRSlotBytes) + gt * 4;
+      unsigned mx = 0;
+#pragma unroll
+      for (int q = 0; q < kRows; ++q) {
+        if (q * kRowElems + gt * 4 < count) {
+          const float4 g4 = *reinterpret_cast<const float4*>(su + q * kRowElems);
+          const float4 e4 = *reinterpret_cast<const float4*>(se + q * kRowElems);
+          const float4 u4 = make_float4(__fadd_rn(g4.x, e4.x), __fadd_rn(g4.y, e4.y), __fadd_rn(g4.z, e4.z),
+                                        __fadd_rn(g4.w, e4.w));
+          *reinterpret_cast<float4*>(su + q * kRowElems) = u4;
+          mx = max(mx, __float_as_uint(fabsf(u4.x)));
+          mx = max(mx, __float_as_uint(fabsf(u4.y)));
+          mx = max(mx, __float_as_uint(fabsf(u4.z)));
+          mx = max(mx, __float_as_uint(fabsf(u4.w)));
+        }
+      }
+      const unsigned wm = warp_max(mx);
+      if (lane == 0 && wm) atomicMax(&hdp->max_bits, wm);
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&ps->e_empty[s]);                            // e has been read: the stage can be refilled
+        mbar_arrive(&ps->hd_ready[i & (kRHeaders - 1)]);         // the header's maximum is complete
+      }
+      if (++s == estages) { s = 0; ph ^= 1u; }
+    }
+  } else {
+    // ------------------------------------------------------------------ store side: quantize, pack, e'
+    // thread (row group, column): rows row0, row0 + kRQRowStep, ... of the tile, 4 elements at column gt
+    const int gt = (tid - kRGroupThreads) & (kRGroupThreads - 1);    // 0..255
+    const int row0 = (tid - kRGroupThreads) / kRGroupThreads;
+    const int gwarp = gt >> 5;
+    int cs = 0;
+    unsigned cph = 0;
+    for (long long i = 0; i < my_tiles; ++i) {
+      if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->cmd_full[cs], cph, abort_flag, p.status))) break;
+      const RCommand cd = ps->cmd[cs];
+      float* su = reinterpret_cast<float*>(slot_base + (size_t)cd.slot * kRSlotBytes) + gt * 4;
+      const float sc = __uint_as_float(cd.scale_bits);
+      unsigned char* cw = p.gcodes + (long long)cd.worker * p.gcode_bytes;
+#pragma unroll
+      for (int q = row0; q < kRows; q += kRQRowStep) {
+        if (q * kRowElems + gt * 4 >= cd.count) continue;              // warp-uniform
+        const float4 u4 = *reinterpret_cast<const float4*>(su + q * kRowElems);
+        const float uu[4] = {u4.x, u4.y, u4.z, u4.w};
+        unsigned code[4];
+        float en[4];
+#pragma unroll
+        for (int c = 0; c < 4; ++c) code[c] = quantize_grad<MODE>(uu[c], sc, p.k, p.L, en[c]);
+        *reinterpret_cast<float4*>(su + q * kRowElems) = make_float4(en[0], en[1], en[2], en[3]);
+        const long long row_elem = cd.off + q * kRowElems + gwarp * 128;
+        void* dst = cw + row_elem * p.bits / 8;
+        if constexpr (MODE == G_TERNARY) {
+          pack_row_store<2>(code[0], code[1], code[2], code[3], dst, lane);
+        } else if constexpr (MODE == G_FIVE) {
+          pack_row_store<3>(code[0], code[1], code[2], code[3], dst, lane);
+        } else {
+          pack_row_store_rt(p.bits, code[0], code[1], code[2], code[3], dst, lane);
+        }
+      }
+      fence_async_shared();                  // e' before the storer's bulk read
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ps->cmd_computed[cs]);
+      if (++cs == kRCmds) { cs = 0; cph ^= 1u; }
+    }
+  }
+  __syncthreads();
+}
+
+}  // namespace qadam
