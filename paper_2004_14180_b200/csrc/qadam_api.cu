@@ -13,7 +13,6 @@
 
 #include "qadam_kernels.cuh"
 #include "qadam_server_pipe.cuh"
-#include "qadam_worker_pipe.cuh"
 #include "qadam_worker_resident.cuh"
 
 #include <cstdlib>
@@ -58,13 +57,8 @@ struct Geometry {
   int gbits = 0, xbits = 0, L = 0;
   GMode gmode = G_TERNARY;
   size_t gcode_bytes = 0, wcode_bytes = 0, workspace_bytes = 0;
-  // fused worker kernel: work items in the order P1(G0) P1(G1) P2(G0) P1(G2) P2(G1) ...
-  std::vector<Run> runs;
   std::vector<int> seg_tiles;        // tiles per segment
-  long long fused_items = 0;
-  long long one_pass_elems = 0;      // padded (worker, element) pairs in groups that fit the L2 budget
-  long long two_pass_elems = 0;      // ... in pairs larger than a group
-  size_t off_ptiles = 0, off_runs = 0, off_done = 0;
+  size_t off_ptiles = 0, off_done = 0;
   // on-chip worker kernel: tiles of the segments that fit on chip (one vector) and the tiles
   // of the remaining segments (two streaming passes)
   std::vector<RTile> rtiles;
@@ -89,93 +83,6 @@ void build_resident(long long capacity, Geometry* g) {
       g->btiles.push_back(t);
     }
   }
-}
-
-// Bytes of g + e (server moments) or g, m, v, e + the u written back (worker moments)
-// that one group of (worker, segment) pairs may hold: a few groups must fit in L2
-// together with what phase 2 writes.
-size_t fused_group_bytes() {
-  const char* env = std::getenv("QADAM_FUSED_GROUP_MB");
-  const long mb = env ? std::atol(env) : 20;
-  return (size_t)(mb > 0 ? mb : 20) << 20;
-}
-
-// Builds the run list of the fused worker kernel for all n workers.
-void build_runs(const qadam_config* c, Geometry* g) {
-  const int S = c->num_segments;
-  g->seg_tiles.assign(S, 0);
-  for (size_t t = 0; t < g->tiles.size(); ++t) g->seg_tiles[g->tiles[t].seg] += 1;
-  const size_t per_elem = c->placement == QADAM_PLACE_WORKER ? 20 : 8;
-  const size_t budget = fused_group_bytes();
-  struct Pair { int worker, seg; };
-  std::vector<std::vector<Pair>> groups;
-  std::vector<bool> solo;
-  size_t cur = 0;
-  for (int w = 0; w < c->n; ++w) {
-    for (int sgm = 0; sgm < S; ++sgm) {
-      const size_t bytes = (size_t)round_up64(g->seg_len[sgm], kAlign) * per_elem;
-      if (bytes > budget) {                       // larger than a group: on its own, two passes over HBM
-        groups.push_back({Pair{w, sgm}});
-        solo.push_back(true);
-        cur = 0;
-        g->two_pass_elems += round_up64(g->seg_len[sgm], kAlign);
-        continue;
-      }
-      if (groups.empty() || solo.back() || cur + bytes > budget) {
-        groups.push_back({});
-        solo.push_back(false);
-        cur = 0;
-      }
-      groups.back().push_back(Pair{w, sgm});
-      cur += bytes;
-      g->one_pass_elems += round_up64(g->seg_len[sgm], kAlign);
-    }
-  }
-  g->runs.clear();
-  long long item = 0;
-  const char* sk_env = std::getenv("QADAM_SOLO_KEEP");
-  const char* sb_env = std::getenv("QADAM_SOLO_BACK");
-  const bool solo_keep = sk_env ? std::atoi(sk_env) != 0 : true;
-  const bool solo_back = sb_env ? std::atoi(sb_env) != 0 : true;
-  auto emit = [&](size_t gi, int phase) {
-    for (const Pair& pr : groups[gi]) {
-      Run r;
-      r.first_item = item;
-      r.seg_off = g->seg_off[pr.seg];
-      r.plen = (int)round_up64(g->seg_len[pr.seg], kAlign);
-      r.ntiles = g->seg_tiles[pr.seg];
-      r.worker = pr.worker;
-      r.seg = pr.seg;
-      r.phase = phase;
-      r.dir = (phase == 1 && solo[gi] && solo_back) ? -1 : 1;   // a lone big pair: phase 2 walks back over the cached tail
-      r.keep = (phase == 0 && (!solo[gi] || solo_keep)) ? 1 : 0;
-      r.pad = 0;
-      g->runs.push_back(r);
-      item += r.ntiles;
-    }
-  };
-  // Phase 2 of a group follows phase 1 of the group `lag` places later: by then every CTA
-  // has pushed the group's phase-1 tiles through its pipeline, so phase 2 does not wait,
-  // and the group (lag + 1 groups in all) is still in L2.  A lone big pair gains nothing
-  // from that (it sweeps L2 anyway): what is owed is finished before it, and it is
-  // finished at once.
-  const char* lag_env = std::getenv("QADAM_FUSED_LAG");
-  const int lag = std::max(1, lag_env ? std::atoi(lag_env) : 1);
-  std::vector<size_t> owed;                          // groups whose phase 2 is still to be emitted
-  size_t owed_head = 0;
-  for (size_t gi = 0; gi < groups.size(); ++gi) {
-    if (solo[gi]) {
-      while (owed_head < owed.size()) emit(owed[owed_head++], 1);
-      emit(gi, 0);
-      emit(gi, 1);
-      continue;
-    }
-    emit(gi, 0);
-    owed.push_back(gi);
-    if (owed.size() - owed_head > (size_t)lag) emit(owed[owed_head++], 1);
-  }
-  while (owed_head < owed.size()) emit(owed[owed_head++], 1);
-  g->fused_items = item;
 }
 
 int validate_config(const qadam_config* c) {
@@ -242,12 +149,11 @@ int build_geometry(const qadam_config* c, Geometry* g) {
   g->xbits = c->kx < 0 ? 0 : c->kx + 2;
   g->gcode_bytes = (size_t)(g->D * g->gbits / 8);
   g->wcode_bytes = (size_t)(g->D * g->xbits / 8);
-  build_runs(c, g);
+  g->seg_tiles.assign(S, 0);
+  for (const Tile& t : g->tiles) g->seg_tiles[t.seg] += 1;
   size_t wo = (size_t)round_up64((int64_t)g->tiles.size() * sizeof(Tile), 256);
   g->off_ptiles = wo;
   wo += (size_t)round_up64((int64_t)g->ptiles.size() * sizeof(Tile), 256);
-  g->off_runs = wo;
-  wo += (size_t)round_up64((int64_t)g->runs.size() * sizeof(Run), 256);
   g->off_done = wo;
   wo += (size_t)round_up64((int64_t)c->n * c->num_segments * sizeof(unsigned), 256);
   // upper bounds (the split into resident and other segments is made at creation, on the device's sizes)
@@ -281,12 +187,6 @@ struct qadam_ctx {
   int pipe_skip_16ths = 2;   // zero skipping while at most this many sixteenths of the workers are live
   size_t pipe_smem = 0;
   CUtensorMap codes_map;
-  // pipelined worker kernel (moments on the server, all workers in one call): grid > 0 when in use
-  int grid_fused = 0;
-  int wpipe_stages = 0;
-  int wpipe_chunk = kChunk;
-  size_t wpipe_smem = 0;
-  Run* d_runs = nullptr;
   unsigned* d_done = nullptr;
   // on-chip worker kernel (moments on the server, all workers in one call): grid > 0 when in use
   int grid_resident = 0;
@@ -375,17 +275,6 @@ PipeKernel pick_pipe(const qadam_ctx* c) {
   if (c->geo.gmode == G_TERNARY) return sm ? pick_pipe_n<true, 2>(c->cfg.n) : pick_pipe_n<false, 2>(c->cfg.n);
   // any other grid of at most 8 bits: table decode, worker count at run time
   return sm ? server_pipe_kernel<true, 0, 0> : server_pipe_kernel<false, 0, 0>;
-}
-
-using WorkerPipeKernel = void (*)(const WorkerPipeParams, const int, const int);
-
-WorkerPipeKernel pick_worker_pipe(const qadam_ctx* c) {
-  switch (c->geo.gmode) {
-    case G_TERNARY: return worker_pipe_kernel<G_TERNARY>;
-    case G_FIVE:    return worker_pipe_kernel<G_FIVE>;
-    case G_POW2:    return worker_pipe_kernel<G_POW2>;
-    default:        return worker_pipe_kernel<G_UNIFORM>;
-  }
 }
 
 using WorkerResidentKernel = void (*)(const WorkerResidentParams);
@@ -523,7 +412,6 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
   {
     unsigned char* ws = static_cast<unsigned char*>(b->workspace);
     c->d_ptiles = reinterpret_cast<Tile*>(ws + c->geo.off_ptiles);
-    c->d_runs = reinterpret_cast<Run*>(ws + c->geo.off_runs);
     c->d_done = reinterpret_cast<unsigned*>(ws + c->geo.off_done);
     c->d_rtiles = reinterpret_cast<RTile*>(ws + c->geo.off_rtiles);
     c->d_btiles = reinterpret_cast<Tile*>(ws + c->geo.off_btiles);
@@ -584,36 +472,18 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
   // plain streaming launches, over a tile table of their own.  The on-chip kernel needs
   // every CTA resident at once (its store side waits for other CTAs' load sides): one
   // CTA per SM, launched cooperatively.
-  // QADAM_WORKER_KERNEL=split: streaming launches only; =pipe: the L2-group pipeline.
+  // QADAM_WORKER_KERNEL=split: streaming launches only.
   {
     int coop = 0, max_smem = 0;
     const char* env = std::getenv("QADAM_WORKER_KERNEL");
     const bool want_split = env && std::strcmp(env, "split") == 0;
-    const bool want_pipe = env && std::strcmp(env, "pipe") == 0;
     const bool eligible = !want_split && c->geo.gmode != G_IDENTITY && cfg->placement == QADAM_PLACE_SERVER &&
         cuda_ok(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev)) && coop &&
         cuda_ok(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
-    if (eligible && want_pipe) {
-      int stages = (int)(((size_t)max_smem - wpipe_smem_bytes(0)) / kWStageBytes);
-      stages = std::min(stages, kWMaxStages) / kWGroups * kWGroups;
-      if (stages >= kWGroups) {
-        c->wpipe_stages = stages;
-        const char* ce = std::getenv("QADAM_WORKER_CHUNK");
-        const int cv = ce ? std::atoi(ce) : kChunk;
-        c->wpipe_chunk = cv >= 1 && cv <= 64 ? cv : kChunk;
-        c->wpipe_smem = wpipe_smem_bytes(stages);
-        int per_sm = 0;
-        if (cuda_ok(cudaFuncSetAttribute(pick_worker_pipe(c), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)c->wpipe_smem)) &&
-            cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pick_worker_pipe(c), kWThreads,
-                                                                  c->wpipe_smem)) &&
-            per_sm >= 1)
-          c->grid_fused = c->sm_count;
-      }
-    } else if (eligible) {
+    if (eligible) {
       // the CTA's shared memory: a ring of slots for u and a few stages for e (227 KB: 14 in all)
       const char* ee = std::getenv("QADAM_RESIDENT_ESTAGES");
-      int estages = ee ? std::atoi(ee) : 3;
+      int estages = ee ? std::atoi(ee) : 2;
       estages = std::max(2, std::min(estages, kRMaxEStages));
       const int slots = std::min(((int)max_smem - kRHeadBytes) / kRSlotBytes - estages, kRMaxSlots);
       // a pair may give a CTA at most slots - 2 tiles: the rest of the ring lets the load side
@@ -645,8 +515,6 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
   if (!cuda_ok(cudaMemcpyAsync(c->d_tiles, c->geo.tiles.data(), c->geo.tiles.size() * sizeof(Tile),
                                cudaMemcpyHostToDevice, c->stream)) ||
       !cuda_ok(cudaMemcpyAsync(c->d_ptiles, c->geo.ptiles.data(), c->geo.ptiles.size() * sizeof(Tile),
-                               cudaMemcpyHostToDevice, c->stream)) ||
-      !cuda_ok(cudaMemcpyAsync(c->d_runs, c->geo.runs.data(), c->geo.runs.size() * sizeof(Run),
                                cudaMemcpyHostToDevice, c->stream)) ||
       (c->grid_resident > 0 &&
        (!cuda_ok(cudaMemcpyAsync(c->d_rtiles, c->geo.rtiles.data(), c->geo.rtiles.size() * sizeof(RTile),
@@ -753,30 +621,6 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
       if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
       c->launches += 2;
     }
-  } else if (c->grid_fused > 0 && worker_begin == 0 && worker_count == c->cfg.n && c->lambda == 0.0f) {
-    // (the pipelined kernel does not stage the held weights: with an l2 term the split kernels run)
-    const size_t pairs = (size_t)c->cfg.n * p.S;
-    if (!cuda_ok(cudaMemsetAsync(p.scale_bits, 0, sizeof(unsigned) * pairs, c->stream)) ||
-        !cuda_ok(cudaMemsetAsync(c->d_done, 0, sizeof(unsigned) * pairs, c->stream)))
-      return QADAM_ERR_CUDA;
-    WorkerPipeParams fp;
-    fp.w = p;
-    fp.runs = c->d_runs;
-    fp.done = c->d_done;
-    fp.total_items = c->geo.fused_items;
-    fp.num_runs = (int)c->geo.runs.size();
-    int stages = c->wpipe_stages;
-    int chunk = c->wpipe_chunk;
-    const int grid = (int)std::min<int64_t>(c->grid_fused, (fp.total_items + chunk - 1) / chunk);
-    void* args[] = {&fp, &stages, &chunk};
-    cudaError_t e;
-    {
-      LaunchTimer lt(c, QADAM_K_WORKER_FUSED);
-      e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(pick_worker_pipe(c)), dim3(grid),
-                                      dim3(kWThreads), args, c->wpipe_smem, c->stream);
-    }
-    if (!cuda_ok(e)) return QADAM_ERR_CUDA;
-    c->launches += 1;
   } else {
     if (!cuda_ok(cudaMemsetAsync(p.scale_bits + (size_t)worker_begin * p.S, 0,
                                  sizeof(unsigned) * (size_t)worker_count * p.S, c->stream)))
@@ -907,9 +751,6 @@ int qadam_worker_pass_model(const qadam_ctx* c, int64_t* one_pass, int64_t* two_
   } else if (c->grid_resident > 0) {
     *one_pass = (int64_t)c->cfg.n * c->geo.resident_elems;
     *two_pass = (int64_t)c->cfg.n * (c->geo.D - c->geo.resident_elems);
-  } else if (c->grid_fused > 0) {
-    *one_pass = c->geo.one_pass_elems;
-    *two_pass = c->geo.two_pass_elems;
   } else {
     *one_pass = 0;
     *two_pass = (int64_t)c->cfg.n * c->geo.D;

@@ -36,9 +36,17 @@
 // the TIMEOUT bit of the status word is set and every role leaves its loop.
 #pragma once
 
-#include "qadam_worker_pipe.cuh"
+#include "qadam_server_pipe.cuh"
 
 namespace qadam {
+
+constexpr unsigned kWSpinLimit = 1u << 21;     // polls of a pair record before giving up
+
+__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 
 // A tile of a resident segment (padded layout, one vector).
 struct __align__(8) RTile {
