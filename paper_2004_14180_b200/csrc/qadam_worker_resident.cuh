@@ -20,9 +20,9 @@
 //                add e to g in place and fold max |u|; a publisher warp adds the CTA's
 //                maximum and tile count to the pair's global record;
 //   store side   a dispatcher warp waits until all tiles of the pair have been counted
-//                (every CTA's, hence the final scale), sixteen consumer warps quantize the
-//                slot, write the packed codes and leave e' in the slot; a storer warp
-//                sends e' back with a bulk store and frees the slot.
+//                (every CTA's, hence the final scale); sixteen consumer warps take u out of
+//                the slot into registers, free the slot at once, quantize, and write the
+//                packed codes and e' straight to global memory.
 // The two sides run as independent loops over the CTA's tiles, coupled only by the
 // pair records in global memory and the slots' "free" barriers: the load side runs
 // ahead of the store side by as many tiles as there are slots, which is what hides the
@@ -73,8 +73,8 @@ struct WorkerResidentParams {
 constexpr int kRGroupThreads = 256;     // load-side consumers: 8 warps, 4 rows of 1024 elements per tile
 constexpr int kRQWarps = QADAM_RESIDENT_QWARPS;   // store-side consumers: 8 or 16 warps (4 or 2 rows per thread)
 constexpr int kRQRowStep = kRQWarps / 8;
-constexpr int kRRoleWarp0 = 8 + kRQWarps;         // producer, publisher, dispatcher, storer follow
-constexpr int kRThreads = 32 * (kRRoleWarp0 + 4);
+constexpr int kRRoleWarp0 = 8 + kRQWarps;         // producer, publisher, dispatcher follow
+constexpr int kRThreads = 32 * (kRRoleWarp0 + 3);
 static_assert(kRQWarps == 8 || kRQWarps == 16, "store-side consumer warps");
 constexpr int kRSlotBytes = kTileElems * 4;
 constexpr int kRCmds = 4;               // quantize commands in flight
@@ -104,7 +104,6 @@ struct RSmem {
   unsigned long long hd_ready[kRHeaders];     // consumers -> publisher: the tile's maximum is in its header
   unsigned long long slot_free[kRMaxSlots];
   unsigned long long cmd_full[kRCmds];
-  unsigned long long cmd_computed[kRCmds];
   unsigned long long cmd_empty[kRCmds];
   RLoadHeader load_hd[kRHeaders];
   RCommand cmd[kRCmds];
@@ -135,11 +134,10 @@ worker_resident_kernel(const WorkerResidentParams rp) {
       mbar_init(&ps->e_empty[s], kRGroupThreads / 32);
     }
     for (int s = 0; s < kRHeaders; ++s) mbar_init(&ps->hd_ready[s], kRGroupThreads / 32);
-    for (int s = 0; s < rp.slots; ++s) mbar_init(&ps->slot_free[s], 1);
+    for (int s = 0; s < rp.slots; ++s) mbar_init(&ps->slot_free[s], kRQWarps);
     for (int s = 0; s < kRCmds; ++s) {
       mbar_init(&ps->cmd_full[s], 1);
-      mbar_init(&ps->cmd_computed[s], kRQWarps);
-      mbar_init(&ps->cmd_empty[s], 1);
+      mbar_init(&ps->cmd_empty[s], kRQWarps);
     }
     ps->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -280,39 +278,6 @@ worker_resident_kernel(const WorkerResidentParams rp) {
         while (j >= rp.TR) { j -= rp.TR; ++worker; }
       }
     }
-  } else if (warp == kRRoleWarp0 + 3) {
-    // ------------------------------------------------------------------ store side: storer
-    int cs = 0;
-    unsigned cph = 0;
-    int owed_slot = -1;                      // slot of the last e' store, not yet freed
-    if (lane == 0) {
-      for (long long i = 0; i < my_tiles; ++i) {
-        if (!mbar_wait_bounded(&ps->cmd_computed[cs], cph, abort_flag, p.status)) break;
-        const RCommand cd = ps->cmd[cs];
-        mbar_arrive(&ps->cmd_empty[cs]);
-        bulk_store(p.e + (long long)cd.worker * p.D + cd.off, slot_base + (size_t)cd.slot * kRSlotBytes,
-                   (unsigned)cd.count * 4u);
-        bulk_commit();
-        if (++cs == kRCmds) { cs = 0; cph ^= 1u; }
-        // A slot is freed once the copy engine has read it.  If the next tile is ready, that
-        // wait is put off by one store so that this warp does not sit in it; if not, there
-        // is nothing better to do than to wait here.
-        const bool next_ready = i + 1 < my_tiles && mbar_try_wait(&ps->cmd_computed[cs], cph);
-        if (next_ready) {
-          if (owed_slot >= 0) {
-            bulk_wait_read_1();
-            mbar_arrive(&ps->slot_free[owed_slot]);
-          }
-          owed_slot = cd.slot;
-        } else {
-          bulk_wait_read_all();
-          if (owed_slot >= 0) mbar_arrive(&ps->slot_free[owed_slot]);
-          mbar_arrive(&ps->slot_free[cd.slot]);
-          owed_slot = -1;
-        }
-      }
-      bulk_wait_all();                       // writes are complete before the kernel ends
-    }
   } else if (warp < 8) {
     // ------------------------------------------------------------------ load side: u = g + e, max |u|
     const int gt = tid;                      // 0..255
@@ -354,24 +319,39 @@ worker_resident_kernel(const WorkerResidentParams rp) {
     const int gt = (tid - kRGroupThreads) & (kRGroupThreads - 1);    // 0..255
     const int row0 = (tid - kRGroupThreads) / kRGroupThreads;
     const int gwarp = gt >> 5;
+    constexpr int kMine = kRows / kRQRowStep;                          // rows per thread
     int cs = 0;
     unsigned cph = 0;
     for (long long i = 0; i < my_tiles; ++i) {
       if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->cmd_full[cs], cph, abort_flag, p.status))) break;
       const RCommand cd = ps->cmd[cs];
-      float* su = reinterpret_cast<float*>(slot_base + (size_t)cd.slot * kRSlotBytes) + gt * 4;
+      const float* su = reinterpret_cast<const float*>(slot_base + (size_t)cd.slot * kRSlotBytes) + gt * 4;
+      // u into registers; from here on neither the slot nor the command is needed
+      float4 u4[kMine];
+#pragma unroll
+      for (int r = 0; r < kMine; ++r) {
+        const int q = row0 + r * kRQRowStep;
+        u4[r] = q * kRowElems + gt * 4 < cd.count ? *reinterpret_cast<const float4*>(su + q * kRowElems)
+                                                  : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
+      }
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&ps->slot_free[cd.slot]);
+        mbar_arrive(&ps->cmd_empty[cs]);
+      }
       const float sc = __uint_as_float(cd.scale_bits);
       unsigned char* cw = p.gcodes + (long long)cd.worker * p.gcode_bytes;
+      float* ew = p.e + (long long)cd.worker * p.D + cd.off + gt * 4;
 #pragma unroll
-      for (int q = row0; q < kRows; q += kRQRowStep) {
+      for (int r = 0; r < kMine; ++r) {
+        const int q = row0 + r * kRQRowStep;
         if (q * kRowElems + gt * 4 >= cd.count) continue;              // warp-uniform
-        const float4 u4 = *reinterpret_cast<const float4*>(su + q * kRowElems);
-        const float uu[4] = {u4.x, u4.y, u4.z, u4.w};
+        const float uu[4] = {u4[r].x, u4[r].y, u4[r].z, u4[r].w};
         unsigned code[4];
         float en[4];
 #pragma unroll
         for (int c = 0; c < 4; ++c) code[c] = quantize_grad<MODE>(uu[c], sc, p.k, p.L, en[c]);
-        *reinterpret_cast<float4*>(su + q * kRowElems) = make_float4(en[0], en[1], en[2], en[3]);
+        *reinterpret_cast<float4*>(ew + q * kRowElems) = make_float4(en[0], en[1], en[2], en[3]);
         const long long row_elem = cd.off + q * kRowElems + gwarp * 128;
         void* dst = cw + row_elem * p.bits / 8;
         if constexpr (MODE == G_TERNARY) {
@@ -382,9 +362,6 @@ worker_resident_kernel(const WorkerResidentParams rp) {
           pack_row_store_rt(p.bits, code[0], code[1], code[2], code[3], dst, lane);
         }
       }
-      fence_async_shared();                  // e' before the storer's bulk read
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&ps->cmd_computed[cs]);
       if (++cs == kRCmds) { cs = 0; cph ^= 1u; }
     }
   }
