@@ -153,24 +153,20 @@ class ClockSampler:
 # ----------------------------------------------------------------------------- byte accounting
 
 def algorithmic_bytes(kernel: str, w, placement: str, D: int, gbits: int, xbits: int,
-                      pass_model=None, l2_term: bool = False, fused_covers_all=None) -> float:
+                      pass_model=None, l2_term: bool = False) -> float:
     """Bytes one launch of `kernel` must move at its interface (fp32 state it has
-    to read and write, packed codes), for all n workers.  For the fused worker kernel
-    the figure is capacity aware: (worker, segment) pairs that fit the kernel's L2
-    group budget are counted once (one pass), larger ones twice (the max-abs scale
-    needs the whole pair before any of it can be quantized)."""
+    to read and write, packed codes), for all n workers.  The worker side is capacity
+    aware: (worker, segment) pairs that fit on chip go through the fused kernel and are
+    counted once (one pass); larger ones take the two streaming launches and are counted
+    twice (the max-abs scale needs the whole pair before any of it can be quantized)."""
     n = w.n
     server_moments = placement == "server"
     # with the l2 term a worker also reads the weights it holds: the packed broadcast, or x
     held = ((xbits / 8.0) if xbits else 4.0) if l2_term else 0.0
-    if kernel == "worker_fused":
-        one_pass, two_pass = pass_model
-        if fused_covers_all is False:   # the on-chip kernel: one-pass pairs only
-            return one_pass * (12.0 + gbits / 8.0)
-        if server_moments:      # read g, e (twice when two-pass); write e and the codes
-            return one_pass * (12.0 + gbits / 8.0) + two_pass * (20.0 + gbits / 8.0)
-        # read g, m, v, e; write m, v, e and codes; two-pass adds a write and a read of u
-        return one_pass * (28.0 + gbits / 8.0) + two_pass * (36.0 + gbits / 8.0)
+    if kernel == "worker_fused":    # the on-chip kernel: the one-pass pairs, every array touched once
+        one_pass, _ = pass_model
+        # read g, e, write e and the codes; moments on the workers: also read and write m, v
+        return one_pass * ((12.0 if server_moments else 28.0) + gbits / 8.0)
     # the split launches cover everything, or, beside the fused kernel, the two-pass pairs only
     split_units = pass_model[1] if pass_model and pass_model[0] > 0 else n * D
     if kernel == "absmax":      # phase 1: read g, e (worker moments: + read m, v, write m, v, u)
@@ -382,9 +378,7 @@ def run_b200(args):
             continue
         per = ms / cnt
         bytes_ = algorithmic_bytes(name, w, args.placement, D, q.gcode_bytes * 8 // D, q.wcode_bytes * 8 // D,
-                                   pass_model=q.worker_pass_model(), l2_term=args.weight_decay != 0.0,
-                                   fused_covers_all=not ("absmax" in prof and prof["absmax"][1] > 0
-                                                         and "worker_fused" in prof and prof["worker_fused"][1] > 0))
+                                   pass_model=q.worker_pass_model(), l2_term=args.weight_decay != 0.0)
         kernels[name] = {"launches": int(cnt), "ms_per_launch": per,
                          "share": ms / sum(m for m, c in prof.values()),
                          "algorithmic_bytes": bytes_, "achieved_gbs": bytes_ / (per * 1e-3) / 1e9,

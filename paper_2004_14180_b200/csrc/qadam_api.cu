@@ -280,11 +280,12 @@ PipeKernel pick_pipe(const qadam_ctx* c) {
 using WorkerResidentKernel = void (*)(const WorkerResidentParams);
 
 WorkerResidentKernel pick_worker_resident(const qadam_ctx* c) {
+  const bool w = c->cfg.placement == QADAM_PLACE_WORKER;
   switch (c->geo.gmode) {
-    case G_TERNARY: return worker_resident_kernel<G_TERNARY>;
-    case G_FIVE:    return worker_resident_kernel<G_FIVE>;
-    case G_POW2:    return worker_resident_kernel<G_POW2>;
-    default:        return worker_resident_kernel<G_UNIFORM>;
+    case G_TERNARY: return w ? worker_resident_kernel<G_TERNARY, true> : worker_resident_kernel<G_TERNARY, false>;
+    case G_FIVE:    return w ? worker_resident_kernel<G_FIVE, true>    : worker_resident_kernel<G_FIVE, false>;
+    case G_POW2:    return w ? worker_resident_kernel<G_POW2, true>    : worker_resident_kernel<G_POW2, false>;
+    default:        return w ? worker_resident_kernel<G_UNIFORM, true> : worker_resident_kernel<G_UNIFORM, false>;
   }
 }
 
@@ -477,7 +478,8 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
     int coop = 0, max_smem = 0;
     const char* env = std::getenv("QADAM_WORKER_KERNEL");
     const bool want_split = env && std::strcmp(env, "split") == 0;
-    const bool eligible = !want_split && c->geo.gmode != G_IDENTITY && cfg->placement == QADAM_PLACE_SERVER &&
+    const bool wm = cfg->placement == QADAM_PLACE_WORKER;
+    const bool eligible = !want_split && c->geo.gmode != G_IDENTITY &&
         cuda_ok(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev)) && coop &&
         cuda_ok(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
     if (eligible) {
@@ -485,7 +487,8 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
       const char* ee = std::getenv("QADAM_RESIDENT_ESTAGES");
       int estages = ee ? std::atoi(ee) : 2;
       estages = std::max(2, std::min(estages, kRMaxEStages));
-      const int slots = std::min(((int)max_smem - kRHeadBytes) / kRSlotBytes - estages, kRMaxSlots);
+      const int slots = std::min(((int)max_smem - kRHeadBytes - estages * resident_stage_bytes(wm)) / kRSlotBytes,
+                                 kRMaxSlots);
       // a pair may give a CTA at most slots - 2 tiles: the rest of the ring lets the load side
       // run ahead into the next pair while this one is quantized and stored
       const char* me = std::getenv("QADAM_RESIDENT_SPARE");
@@ -494,7 +497,7 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
         build_resident((long long)c->sm_count * (slots - spare), &c->geo);
         c->res_slots = slots;
         c->res_estages = estages;
-        c->res_smem = resident_smem_bytes(slots, estages);
+        c->res_smem = resident_smem_bytes(slots, estages, wm);
         int per_sm = 0;
         if (!c->geo.rtiles.empty() &&
             cuda_ok(cudaFuncSetAttribute(pick_worker_resident(c), cudaFuncAttributeMaxDynamicSharedMemorySize,

@@ -67,15 +67,16 @@ struct WorkerResidentParams {
   int estages;            // stages of the e ring
 };
 
-#ifndef QADAM_RESIDENT_QWARPS
-#define QADAM_RESIDENT_QWARPS 16
-#endif
-constexpr int kRGroupThreads = 256;     // load-side consumers: 8 warps, 4 rows of 1024 elements per tile
-constexpr int kRQWarps = QADAM_RESIDENT_QWARPS;   // store-side consumers: 8 or 16 warps (4 or 2 rows per thread)
-constexpr int kRQRowStep = kRQWarps / 8;
-constexpr int kRRoleWarp0 = 8 + kRQWarps;         // producer, publisher, dispatcher follow
+// 24 consumer warps, split between the two sides by where the arithmetic is: with the
+// moments on the server the load side only adds (8 warps, 4 rows of 1024 elements per
+// thread and tile) and the store side quantizes (16 warps, 2 rows); with the moments on
+// the workers the load side also runs the moment updates, a root and a division per
+// element (16 warps) and the store side gets 8.
+constexpr int kRColThreads = 256;       // threads across a 1024-element row, 4 elements each
+constexpr int kRConsumerWarps = 24;
+constexpr int kRRoleWarp0 = kRConsumerWarps;      // producer, publisher, dispatcher follow
 constexpr int kRThreads = 32 * (kRRoleWarp0 + 3);
-static_assert(kRQWarps == 8 || kRQWarps == 16, "store-side consumer warps");
+__host__ __device__ constexpr int resident_load_warps(bool worker_moments) { return worker_moments ? 16 : 8; }
 constexpr int kRSlotBytes = kTileElems * 4;
 constexpr int kRCmds = 4;               // quantize commands in flight
 constexpr int kRMaxEStages = 8;
@@ -89,6 +90,7 @@ struct RLoadHeader {       // one per tile in flight on the load side (ring of k
   int count;               // elements of the tile
   int publish;             // last tile of the CTA's streak of this pair
   unsigned max_bits;       // max |u| of the tile, folded in by the consumer warps
+  long long elem;          // worker * D + first element: where m, v go back (moments on the workers)
 };
 struct RCommand {          // one per quantize command
   long long off;           // first element (padded layout)
@@ -111,13 +113,21 @@ struct RSmem {
 };
 static_assert(sizeof(RSmem) <= kRHeadBytes, "head of the shared-memory layout");
 
-__host__ __device__ inline size_t resident_smem_bytes(int slots, int estages) {
-  return kRHeadBytes + (size_t)(slots + estages) * kRSlotBytes;
+// A stage of the ring holds the tile's e, and with the moments on the workers its m and v.
+__host__ __device__ constexpr int resident_stage_bytes(bool worker_moments) {
+  return (worker_moments ? 3 : 1) * kRSlotBytes;
+}
+__host__ __device__ inline size_t resident_smem_bytes(int slots, int estages, bool worker_moments) {
+  return kRHeadBytes + (size_t)slots * kRSlotBytes + (size_t)estages * resident_stage_bytes(worker_moments);
 }
 
-template <int MODE>
+template <int MODE, bool WM>
 __global__ void __launch_bounds__(kRThreads, 1)
 worker_resident_kernel(const WorkerResidentParams rp) {
+  constexpr int kLWarps = resident_load_warps(WM);          // load-side consumer warps
+  constexpr int kQWarps = kRConsumerWarps - kLWarps;        // store-side consumer warps
+  constexpr int kLRowStep = kLWarps / 8, kQRowStep = kQWarps / 8;
+  constexpr int kStageBytes = resident_stage_bytes(WM);
   extern __shared__ __align__(128) unsigned char smem_raw[];
   RSmem* ps = reinterpret_cast<RSmem*>(smem_raw);
   unsigned char* slot_base = smem_raw + kRHeadBytes;
@@ -131,13 +141,13 @@ worker_resident_kernel(const WorkerResidentParams rp) {
   if (tid == 0) {
     for (int s = 0; s < estages; ++s) {
       mbar_init(&ps->e_full[s], 1);
-      mbar_init(&ps->e_empty[s], kRGroupThreads / 32);
+      mbar_init(&ps->e_empty[s], kLWarps);
     }
-    for (int s = 0; s < kRHeaders; ++s) mbar_init(&ps->hd_ready[s], kRGroupThreads / 32);
-    for (int s = 0; s < rp.slots; ++s) mbar_init(&ps->slot_free[s], kRQWarps);
+    for (int s = 0; s < kRHeaders; ++s) mbar_init(&ps->hd_ready[s], kLWarps);
+    for (int s = 0; s < rp.slots; ++s) mbar_init(&ps->slot_free[s], kQWarps);
     for (int s = 0; s < kRCmds; ++s) {
       mbar_init(&ps->cmd_full[s], 1);
-      mbar_init(&ps->cmd_empty[s], kRQWarps);
+      mbar_init(&ps->cmd_empty[s], kQWarps);
     }
     ps->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -181,9 +191,15 @@ worker_resident_kernel(const WorkerResidentParams rp) {
           hd->max_bits = 0u;
           const unsigned bytes = (unsigned)cur.count * 4u;
           const long long eo = (long long)worker * p.D + cur.off;
-          mbar_arrive_expect_tx(&ps->e_full[s], 2u * bytes);
+          hd->elem = eo;
+          unsigned char* st = ering_base + (size_t)s * kStageBytes;
+          mbar_arrive_expect_tx(&ps->e_full[s], (WM ? 4u : 2u) * bytes);
           bulk_load(slot_base + (size_t)slot * kRSlotBytes, p.g + eo, bytes, &ps->e_full[s]);
-          bulk_load(ering_base + (size_t)s * kRSlotBytes, p.e + eo, bytes, &ps->e_full[s]);
+          bulk_load(st, p.e + eo, bytes, &ps->e_full[s]);
+          if constexpr (WM) {
+            bulk_load(st + kRSlotBytes, p.m + eo, bytes, &ps->e_full[s]);
+            bulk_load(st + 2 * kRSlotBytes, p.v + eo, bytes, &ps->e_full[s]);
+          }
         }
       }
       ok = __shfl_sync(0xffffffffu, ok, 0);
@@ -278,9 +294,11 @@ worker_resident_kernel(const WorkerResidentParams rp) {
         while (j >= rp.TR) { j -= rp.TR; ++worker; }
       }
     }
-  } else if (warp < 8) {
-    // ------------------------------------------------------------------ load side: u = g + e, max |u|
-    const int gt = tid;                      // 0..255
+  } else if (warp < kLWarps) {
+    // ------------------------------------------------------------------ load side: u into the slot, max |u|
+    // thread (row group, column): rows row0, row0 + kLRowStep, ... of the tile, 4 elements at column gt
+    const int gt = tid & (kRColThreads - 1);
+    const int row0 = tid / kRColThreads;
     int s = 0;
     unsigned ph = 0;
     for (long long i = 0; i < my_tiles; ++i) {
@@ -288,38 +306,74 @@ worker_resident_kernel(const WorkerResidentParams rp) {
       RLoadHeader* hdp = &ps->load_hd[i & (kRHeaders - 1)];
       const int slot = hdp->slot, count = hdp->count;
       float* su = reinterpret_cast<float*>(slot_base + (size_t)slot * kRSlotBytes) + gt * 4;
-      const float* se = reinterpret_cast<const float*>(ering_base + (size_t)s * kRSlotBytes) + gt * 4;
+      const float* se = reinterpret_cast<const float*>(ering_base + (size_t)s * kStageBytes) + gt * 4;
       unsigned mx = 0;
+      if constexpr (WM) {
+        // Algorithm 3: v, m updates, u = alpha m / sqrt(v + eps) + e; m, v go straight back
+        const long long elem = hdp->elem;
+        float4 g4[kRows / kLRowStep], e4[kRows / kLRowStep], m4[kRows / kLRowStep], v4[kRows / kLRowStep];
 #pragma unroll
-      for (int q = 0; q < kRows; ++q) {
-        if (q * kRowElems + gt * 4 < count) {
-          const float4 g4 = *reinterpret_cast<const float4*>(su + q * kRowElems);
-          const float4 e4 = *reinterpret_cast<const float4*>(se + q * kRowElems);
-          const float4 u4 = make_float4(__fadd_rn(g4.x, e4.x), __fadd_rn(g4.y, e4.y), __fadd_rn(g4.z, e4.z),
-                                        __fadd_rn(g4.w, e4.w));
-          *reinterpret_cast<float4*>(su + q * kRowElems) = u4;
-          mx = max(mx, __float_as_uint(fabsf(u4.x)));
-          mx = max(mx, __float_as_uint(fabsf(u4.y)));
-          mx = max(mx, __float_as_uint(fabsf(u4.z)));
-          mx = max(mx, __float_as_uint(fabsf(u4.w)));
+        for (int r = 0; r < kRows / kLRowStep; ++r) {
+          const int q = row0 + r * kLRowStep;
+          if (q * kRowElems + gt * 4 < count) {
+            g4[r] = *reinterpret_cast<const float4*>(su + q * kRowElems);
+            e4[r] = *reinterpret_cast<const float4*>(se + q * kRowElems);
+            m4[r] = *reinterpret_cast<const float4*>(se + kTileElems + q * kRowElems);
+            v4[r] = *reinterpret_cast<const float4*>(se + 2 * kTileElems + q * kRowElems);
+          }
+        }
+#pragma unroll
+        for (int r = 0; r < kRows / kLRowStep; ++r) {
+          const int q = row0 + r * kLRowStep;
+          if (q * kRowElems + gt * 4 >= count) continue;               // warp-uniform
+          float gg[4] = {g4[r].x, g4[r].y, g4[r].z, g4[r].w};
+          float ee[4] = {e4[r].x, e4[r].y, e4[r].z, e4[r].w};
+          float mm[4] = {m4[r].x, m4[r].y, m4[r].z, m4[r].w};
+          float vs[4] = {v4[r].x, v4[r].y, v4[r].z, v4[r].w};
+          float uu[4];
+#pragma unroll
+          for (int c = 0; c < 4; ++c) {
+            moments(p.h, gg[c], mm[c], vs[c]);
+            uu[c] = __fadd_rn(adam_step(p.h, mm[c], vs[c], p.alpha), ee[c]);
+            mx = max(mx, __float_as_uint(fabsf(uu[c])));
+          }
+          *reinterpret_cast<float4*>(su + q * kRowElems) = make_float4(uu[0], uu[1], uu[2], uu[3]);
+          const long long o = elem + q * kRowElems + gt * 4;
+          *reinterpret_cast<float4*>(p.m + o) = make_float4(mm[0], mm[1], mm[2], mm[3]);
+          *reinterpret_cast<float4*>(p.v + o) = make_float4(vs[0], vs[1], vs[2], vs[3]);
+        }
+      } else {
+#pragma unroll
+        for (int q = row0; q < kRows; q += kLRowStep) {
+          if (q * kRowElems + gt * 4 < count) {
+            const float4 g4 = *reinterpret_cast<const float4*>(su + q * kRowElems);
+            const float4 e4 = *reinterpret_cast<const float4*>(se + q * kRowElems);
+            const float4 u4 = make_float4(__fadd_rn(g4.x, e4.x), __fadd_rn(g4.y, e4.y), __fadd_rn(g4.z, e4.z),
+                                          __fadd_rn(g4.w, e4.w));
+            *reinterpret_cast<float4*>(su + q * kRowElems) = u4;
+            mx = max(mx, __float_as_uint(fabsf(u4.x)));
+            mx = max(mx, __float_as_uint(fabsf(u4.y)));
+            mx = max(mx, __float_as_uint(fabsf(u4.z)));
+            mx = max(mx, __float_as_uint(fabsf(u4.w)));
+          }
         }
       }
       const unsigned wm = warp_max(mx);
       if (lane == 0 && wm) atomicMax(&hdp->max_bits, wm);
       __syncwarp();
       if (lane == 0) {
-        mbar_arrive(&ps->e_empty[s]);                            // e has been read: the stage can be refilled
+        mbar_arrive(&ps->e_empty[s]);                            // the stage has been read: it can be refilled
         mbar_arrive(&ps->hd_ready[i & (kRHeaders - 1)]);         // the header's maximum is complete
       }
       if (++s == estages) { s = 0; ph ^= 1u; }
     }
   } else {
     // ------------------------------------------------------------------ store side: quantize, pack, e'
-    // thread (row group, column): rows row0, row0 + kRQRowStep, ... of the tile, 4 elements at column gt
-    const int gt = (tid - kRGroupThreads) & (kRGroupThreads - 1);    // 0..255
-    const int row0 = (tid - kRGroupThreads) / kRGroupThreads;
+    // thread (row group, column): rows row0, row0 + kQRowStep, ... of the tile, 4 elements at column gt
+    const int gt = (tid - 32 * kLWarps) & (kRColThreads - 1);          // 0..255
+    const int row0 = (tid - 32 * kLWarps) / kRColThreads;
     const int gwarp = gt >> 5;
-    constexpr int kMine = kRows / kRQRowStep;                          // rows per thread
+    constexpr int kMine = kRows / kQRowStep;                            // rows per thread
     int cs = 0;
     unsigned cph = 0;
     for (long long i = 0; i < my_tiles; ++i) {
@@ -330,7 +384,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
       float4 u4[kMine];
 #pragma unroll
       for (int r = 0; r < kMine; ++r) {
-        const int q = row0 + r * kRQRowStep;
+        const int q = row0 + r * kQRowStep;
         u4[r] = q * kRowElems + gt * 4 < cd.count ? *reinterpret_cast<const float4*>(su + q * kRowElems)
                                                   : make_float4(0.0f, 0.0f, 0.0f, 0.0f);
       }
@@ -344,7 +398,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
       float* ew = p.e + (long long)cd.worker * p.D + cd.off + gt * 4;
 #pragma unroll
       for (int r = 0; r < kMine; ++r) {
-        const int q = row0 + r * kRQRowStep;
+        const int q = row0 + r * kQRowStep;
         if (q * kRowElems + gt * 4 >= cd.count) continue;              // warp-uniform
         const float uu[4] = {u4[r].x, u4[r].y, u4[r].z, u4[r].w};
         unsigned code[4];

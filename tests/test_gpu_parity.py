@@ -218,43 +218,48 @@ def test_table_decoded_grid_sparse_and_dense_regions():
 
 # ---------------------------------------------------------------- the on-chip worker kernel
 
-def test_on_chip_worker_many_small_tensors():
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_on_chip_worker_many_small_tensors(placement):
     # hundreds of (worker, segment) pairs of one or two tiles: streaks of a single tile,
     # CTAs that own nothing of a pair, pairs that end in the middle of a tile row
     rng = np.random.default_rng(11)
     seg = [int(v) for v in rng.integers(1, 6000, size=400)]
-    _run(seg, 3, 0, 0, S_MODE, T=3, seed=12)
-    _run(seg[:150], 5, 1, 1, S_MODE, T=2, seed=13)
+    _run(seg, 3, 0, 0, placement, T=3, seed=12)
+    _run(seg[:150], 5, 1, 1, placement, T=2, seed=13)
 
 
-def test_on_chip_worker_rings_wrap():
-    # more than 32 tiles per CTA: the rings of slots, e stages and tile headers all go round
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_on_chip_worker_rings_wrap(placement):
+    # more than 32 tiles per CTA: the rings of slots, stages and tile headers all go round
     sms = torch.cuda.get_device_properties(0).multi_processor_count
-    per_seg = sms * 9 * 4096 + 4096 + 300            # 10 tiles for some CTAs, a ragged tail
-    _run([per_seg, 5000, per_seg, 77], 2, 0, 0, S_MODE, T=3, seed=14)
+    per_seg = sms * 5 * 4096 + 4096 + 300            # 6 tiles for some CTAs, a ragged tail
+    _run([per_seg, 5000, per_seg, 77, per_seg], 3, 0, 0, placement, T=3, seed=14)
 
 
-def test_on_chip_worker_capacity_boundary():
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_on_chip_worker_capacity_boundary(placement):
     # tensors around the largest pair the on-chip kernel takes: the kernel and the two
     # streaming launches share one step, each over its own tile table
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     rng = np.random.default_rng(15)
     tile = 4096
-    for slots_used in (10, 11, 12):                  # around slots - spare for a 227 KB SM
+    # around slots - spare for a 227 KB SM: 12 - 2 (moments on the server), 8 - 2 (on the workers)
+    lo = 10 if placement == S_MODE else 6
+    for slots_used in (lo, lo + 1, lo + 2):
         cap = sms * slots_used * tile
         seg = [cap, 300, cap + tile, 70000, cap - tile + 1]
         n, d = 2, sum([cap, 300, cap + tile, 70000, cap - tile + 1])
         x1 = (rng.standard_normal(d) * 0.2).astype(np.float32)
-        p = Pair(seg, n, 0, 0, S_MODE, x1=x1)
+        p = Pair(seg, n, 0, 0, placement, x1=x1)
         one, two = p.gpu.worker_pass_model()
         assert one + two == n * p.gpu.D
         for t in range(2):
             p.step(_rand_grads(rng, n, d))
             p.compare_state()
         p.close()
-        if slots_used == 10:
+        if slots_used == lo:
             assert one > 0, "no pair took the on-chip kernel"
-        if slots_used == 12:
+        if slots_used == lo + 2:
             assert two > 0, "no pair took the streaming launches"
 
 
