@@ -166,7 +166,7 @@ def algorithmic_bytes(kernel: str, w, placement: str, D: int, gbits: int, xbits:
     if kernel == "worker_fused":    # the on-chip kernel: the one-pass pairs, every array touched once
         one_pass, _ = pass_model
         # read g, e, write e and the codes; moments on the workers: also read and write m, v
-        return one_pass * ((12.0 if server_moments else 28.0) + gbits / 8.0)
+        return one_pass * ((12.0 if server_moments else 28.0) + held + gbits / 8.0)
     # the split launches cover everything, or, beside the fused kernel, the two-pass pairs only
     split_units = pass_model[1] if pass_model and pass_model[0] > 0 else n * D
     if kernel == "absmax":      # phase 1: read g, e (worker moments: + read m, v, write m, v, u)

@@ -226,16 +226,18 @@ enum {
   QADAM_K_IDENTITY = 2,    /* worker with Q_g = identity                              */
   QADAM_K_SERVER = 3,      /* fused server pass                                       */
   QADAM_K_BROADCAST = 4,   /* stand-alone Q_x(x_1)                                    */
-  QADAM_K_WORKER_FUSED = 5,/* both worker phases in one persistent kernel             */
+  QADAM_K_WORKER_FUSED = 5,/* both worker phases in one persistent kernel, for the
+                              (worker, segment) pairs that fit on chip                */
   QADAM_NUM_KERNELS = 6
 };
 int qadam_profile_enable(qadam_ctx* ctx, int enable);
 int qadam_profile_read(qadam_ctx* ctx, double* ms, int64_t* launches);
 
-/* Instrumentation: how the worker side of this context moves its data.  one_pass:
- * padded (worker, element) pairs that belong to (worker, segment) pairs small enough
- * to stay in L2 between the two worker phases (read from HBM once); two_pass: pairs
- * in segments too large for that (read twice).  The sum is n * D. */
+/* Instrumentation: how the worker side of this context moves its data when all
+ * workers are compressed in one call.  one_pass: padded (worker, element) pairs that
+ * belong to (worker, segment) pairs small enough to be held on chip between the
+ * max-abs reduction and the quantization (read from HBM once); two_pass: pairs in
+ * segments too large for that (read twice).  The sum is n * D. */
 int qadam_worker_pass_model(const qadam_ctx* ctx, int64_t* one_pass, int64_t* two_pass);
 
 /* Number of kernels this context has launched since it was created. */

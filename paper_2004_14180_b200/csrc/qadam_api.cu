@@ -279,14 +279,29 @@ PipeKernel pick_pipe(const qadam_ctx* c) {
 
 using WorkerResidentKernel = void (*)(const WorkerResidentParams);
 
-WorkerResidentKernel pick_worker_resident(const qadam_ctx* c) {
+template <int MODE>
+WorkerResidentKernel pick_worker_resident_mode(bool worker_moments, bool l2) {
+  if (worker_moments) return l2 ? worker_resident_kernel<MODE, true, true> : worker_resident_kernel<MODE, true, false>;
+  return l2 ? worker_resident_kernel<MODE, false, true> : worker_resident_kernel<MODE, false, false>;
+}
+
+WorkerResidentKernel pick_worker_resident(const qadam_ctx* c, bool l2) {
   const bool w = c->cfg.placement == QADAM_PLACE_WORKER;
   switch (c->geo.gmode) {
-    case G_TERNARY: return w ? worker_resident_kernel<G_TERNARY, true> : worker_resident_kernel<G_TERNARY, false>;
-    case G_FIVE:    return w ? worker_resident_kernel<G_FIVE, true>    : worker_resident_kernel<G_FIVE, false>;
-    case G_POW2:    return w ? worker_resident_kernel<G_POW2, true>    : worker_resident_kernel<G_POW2, false>;
-    default:        return w ? worker_resident_kernel<G_UNIFORM, true> : worker_resident_kernel<G_UNIFORM, false>;
+    case G_TERNARY: return pick_worker_resident_mode<G_TERNARY>(w, l2);
+    case G_FIVE:    return pick_worker_resident_mode<G_FIVE>(w, l2);
+    case G_POW2:    return pick_worker_resident_mode<G_POW2>(w, l2);
+    default:        return pick_worker_resident_mode<G_UNIFORM>(w, l2);
   }
+}
+
+// With the l2 term and the moments on the server the streaming launches run instead of the
+// on-chip kernel: its 8 load-side warps fetch the held weights from global memory with
+// nothing to hide the latency behind, and lose (measured: 6.6 ms against 2.5 + 4.5 ms for
+// everything on the BERT-base-shaped set).  With the moments on the workers the load side
+// has 16 warps and more arithmetic per element, and the on-chip kernel wins.
+bool l2_split(const qadam_ctx* c) {
+  return c->lambda != 0.0f && c->cfg.placement == QADAM_PLACE_SERVER;
 }
 
 // grids of the split worker kernels (they depend on whether the l2 term is on)
@@ -500,9 +515,14 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
         c->res_smem = resident_smem_bytes(slots, estages, wm);
         int per_sm = 0;
         if (!c->geo.rtiles.empty() &&
-            cuda_ok(cudaFuncSetAttribute(pick_worker_resident(c), cudaFuncAttributeMaxDynamicSharedMemorySize,
+            cuda_ok(cudaFuncSetAttribute(pick_worker_resident(c, false), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          (int)c->res_smem)) &&
-            cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pick_worker_resident(c), kRThreads,
+            cuda_ok(cudaFuncSetAttribute(pick_worker_resident(c, true), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         (int)c->res_smem)) &&
+            cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pick_worker_resident(c, false), kRThreads,
+                                                                  c->res_smem)) &&
+            per_sm >= 1 &&
+            cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pick_worker_resident(c, true), kRThreads,
                                                                   c->res_smem)) &&
             per_sm >= 1)
           c->grid_resident = c->sm_count;
@@ -582,8 +602,7 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
     }
     if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
     c->launches += 1;
-  } else if (c->grid_resident > 0 && worker_begin == 0 && worker_count == c->cfg.n && c->lambda == 0.0f) {
-    // (the on-chip kernel does not stage the held weights: with an l2 term the split kernels run)
+  } else if (c->grid_resident > 0 && worker_begin == 0 && worker_count == c->cfg.n && !l2_split(c)) {
     const size_t pairs = (size_t)c->cfg.n * p.S;
     if (!cuda_ok(cudaMemsetAsync(p.scale_bits, 0, sizeof(unsigned) * pairs, c->stream)) ||
         !cuda_ok(cudaMemsetAsync(c->d_done, 0, sizeof(unsigned) * pairs, c->stream)))
@@ -600,7 +619,7 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
     cudaError_t e;
     {
       LaunchTimer lt(c, QADAM_K_WORKER_FUSED);
-      e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(pick_worker_resident(c)),
+      e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(pick_worker_resident(c, c->lambda != 0.0f)),
                                       dim3(c->grid_resident), dim3(kRThreads), args, c->res_smem, c->stream);
     }
     if (!cuda_ok(e)) return QADAM_ERR_CUDA;
@@ -748,10 +767,7 @@ int qadam_profile_read(qadam_ctx* c, double* ms, int64_t* launches) {
 
 int qadam_worker_pass_model(const qadam_ctx* c, int64_t* one_pass, int64_t* two_pass) {
   if (!c || !one_pass || !two_pass) return QADAM_ERR_NULL;
-  if (c->lambda != 0.0f) {              // with the l2 term the split launches cover everything
-    *one_pass = 0;
-    *two_pass = (int64_t)c->cfg.n * c->geo.D;
-  } else if (c->grid_resident > 0) {
+  if (c->grid_resident > 0 && !l2_split(c)) {
     *one_pass = (int64_t)c->cfg.n * c->geo.resident_elems;
     *two_pass = (int64_t)c->cfg.n * (c->geo.D - c->geo.resident_elems);
   } else {

@@ -1,27 +1,30 @@
-// The worker side (moments on the server) for tensors that fit ON CHIP: one persistent
-// kernel that reads g and e once, keeps u = g + e in shared memory until the tensor's
-// scale is known, and quantizes from there.
+// The worker side for tensors that fit ON CHIP: one persistent kernel that reads g and e
+// (and, with the moments on the workers, m and v) once, keeps u in shared memory until
+// the tensor's scale is known, and quantizes from there.  u = g + e with the moments on
+// the server, u = alpha m / sqrt(v + eps) + e after the moment updates of Algorithm 3
+// with the moments on the workers.
 //
 // The scale of Q_g is the maximum of |u| over a whole (worker, segment) pair, so no
 // element of a pair can be quantized before all of the pair has been read.  Going back
 // to memory for the second look costs as much through L2 as from HBM on this machine
 // (the path from L2 into an SM carries little more than HBM delivers: measured), so the
 // only way to touch each element once is to hold u where it was computed.  Each of the
-// 148 SMs keeps a ring of 10 to 12 slots of 4096 values; a pair spread over all SMs may
-// therefore be up to a few million elements long.  Per pair and element this moves g, e
-// in and e', the packed code out: 12 + b_g / 8 bytes, the least the method allows.
+// 148 SMs keeps a ring of 12 slots of 4096 values (8 when m and v are staged too); a pair
+// spread over all SMs may therefore be up to a few million elements long.  Per pair and
+// element this moves g, e in and e', the packed code out: 12 + b_g / 8 bytes (28 + b_g / 8
+// with m, v read and written), the least the method allows.
 //
 // The resident tiles of all workers are numbered worker-major, t = worker * TR + j
 // (j: index in the per-vector list of resident tiles), so the tiles of a pair are
 // consecutive.  Tile t belongs to CTA t mod gridDim.x; a CTA takes its tiles in
 // increasing order and its i-th tile lives in slot i mod slots.  Per CTA, one per SM:
-//   load side    a producer warp brings g into the tile's slot and e into a small ring
-//                with bulk copies that complete on an mbarrier; eight consumer warps
-//                add e to g in place and fold max |u|; a publisher warp adds the CTA's
-//                maximum and tile count to the pair's global record;
+//   load side    a producer warp brings g into the tile's slot and e (m, v) into a small
+//                ring with bulk copies that complete on an mbarrier; consumer warps form u
+//                in place, fold max |u| (and write m, v back); a publisher warp adds the
+//                CTA's maximum and tile count to the pair's global record;
 //   store side   a dispatcher warp waits until all tiles of the pair have been counted
-//                (every CTA's, hence the final scale); sixteen consumer warps take u out of
-//                the slot into registers, free the slot at once, quantize, and write the
+//                (every CTA's, hence the final scale); consumer warps take u out of the
+//                slot into registers, free the slot at once, quantize, and write the
 //                packed codes and e' straight to global memory.
 // The two sides run as independent loops over the CTA's tiles, coupled only by the
 // pair records in global memory and the slots' "free" barriers: the load side runs
@@ -91,6 +94,7 @@ struct RLoadHeader {       // one per tile in flight on the load side (ring of k
   int publish;             // last tile of the CTA's streak of this pair
   unsigned max_bits;       // max |u| of the tile, folded in by the consumer warps
   long long elem;          // worker * D + first element: where m, v go back (moments on the workers)
+  long long off;           // first element in the vector: where the held weights are (l2 term)
 };
 struct RCommand {          // one per quantize command
   long long off;           // first element (padded layout)
@@ -121,7 +125,9 @@ __host__ __device__ inline size_t resident_smem_bytes(int slots, int estages, bo
   return kRHeadBytes + (size_t)slots * kRSlotBytes + (size_t)estages * resident_stage_bytes(worker_moments);
 }
 
-template <int MODE, bool WM>
+// MODE: grid of Q_g; WM: moments on the workers; L2: the l2 term lambda * (held weights) is
+// added to g first (the held weights are decoded from the packed broadcast, or read from x).
+template <int MODE, bool WM, bool L2>
 __global__ void __launch_bounds__(kRThreads, 1)
 worker_resident_kernel(const WorkerResidentParams rp) {
   constexpr int kLWarps = resident_load_warps(WM);          // load-side consumer warps
@@ -192,6 +198,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
           const unsigned bytes = (unsigned)cur.count * 4u;
           const long long eo = (long long)worker * p.D + cur.off;
           hd->elem = eo;
+          hd->off = cur.off;
           unsigned char* st = ering_base + (size_t)s * kStageBytes;
           mbar_arrive_expect_tx(&ps->e_full[s], (WM ? 4u : 2u) * bytes);
           bulk_load(slot_base + (size_t)slot * kRSlotBytes, p.g + eo, bytes, &ps->e_full[s]);
@@ -311,6 +318,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
       if constexpr (WM) {
         // Algorithm 3: v, m updates, u = alpha m / sqrt(v + eps) + e; m, v go straight back
         const long long elem = hdp->elem;
+        const long long off = hdp->off;
         float4 g4[kRows / kLRowStep], e4[kRows / kLRowStep], m4[kRows / kLRowStep], v4[kRows / kLRowStep];
 #pragma unroll
         for (int r = 0; r < kRows / kLRowStep; ++r) {
@@ -328,6 +336,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
           if (q * kRowElems + gt * 4 >= count) continue;               // warp-uniform
           float gg[4] = {g4[r].x, g4[r].y, g4[r].z, g4[r].w};
           float ee[4] = {e4[r].x, e4[r].y, e4[r].z, e4[r].w};
+          if constexpr (L2) add_l2_term(p, off + q * kRowElems + (gt >> 5) * 128, lane, gg);
           float mm[4] = {m4[r].x, m4[r].y, m4[r].z, m4[r].w};
           float vs[4] = {v4[r].x, v4[r].y, v4[r].z, v4[r].w};
           float uu[4];
@@ -348,8 +357,10 @@ worker_resident_kernel(const WorkerResidentParams rp) {
           if (q * kRowElems + gt * 4 < count) {
             const float4 g4 = *reinterpret_cast<const float4*>(su + q * kRowElems);
             const float4 e4 = *reinterpret_cast<const float4*>(se + q * kRowElems);
-            const float4 u4 = make_float4(__fadd_rn(g4.x, e4.x), __fadd_rn(g4.y, e4.y), __fadd_rn(g4.z, e4.z),
-                                          __fadd_rn(g4.w, e4.w));
+            float gg[4] = {g4.x, g4.y, g4.z, g4.w};
+            if constexpr (L2) add_l2_term(p, hdp->off + q * kRowElems + (gt >> 5) * 128, lane, gg);
+            const float4 u4 = make_float4(__fadd_rn(gg[0], e4.x), __fadd_rn(gg[1], e4.y), __fadd_rn(gg[2], e4.z),
+                                          __fadd_rn(gg[3], e4.w));
             *reinterpret_cast<float4*>(su + q * kRowElems) = u4;
             mx = max(mx, __float_as_uint(fabsf(u4.x)));
             mx = max(mx, __float_as_uint(fabsf(u4.y)));
