@@ -43,9 +43,13 @@ NCU_TRAFFIC = {
     # kernel: (bytes per unit, digest of csrc/ at capture time)
     # profiles/dram_traffic_flat28_n16_server_moments.txt: the benchmark's own workload
     # (flat28, n = 16, moments on the server), one-pass capture of the two byte counters
-    "absmax": (8.00, "8cd9bfdcf5c36862"),
-    "quantize": (12.24, "8cd9bfdcf5c36862"),
-    "server": (28.03, "8cd9bfdcf5c36862"),
+    "absmax": (8.00, "7a40b2d310420c55"),
+    "quantize": (12.24, "7a40b2d310420c55"),
+    "server": (28.03, "7a40b2d310420c55"),
+    # profiles/worker_resident_bert_base_n4.md: the on-chip worker kernel on the BERT-base-shaped
+    # set with n = 4 (a case small enough for a multi-pass capture), scaled by the pairs it takes
+    "worker_fused:server": (12.12, "7a40b2d310420c55"),
+    "worker_fused:worker": (28.10, "7a40b2d310420c55"),
 }
 
 
@@ -385,9 +389,13 @@ def run_b200(args):
                          "frac": bytes_ / (per * 1e-3) / 1e9 / peak}
     dom = max(kernels, key=lambda k: kernels[k]["launches"] * kernels[k]["ms_per_launch"])
     traffic = None
-    if dom in NCU_TRAFFIC and NCU_TRAFFIC[dom][1] == csrc_digest():
-        units = w.n * D if dom in ("absmax", "quantize", "identity", "worker_fused") else D
-        traffic = NCU_TRAFFIC[dom][0] * units
+    tkey = f"{dom}:{args.placement}" if dom == "worker_fused" else dom
+    if tkey in NCU_TRAFFIC and NCU_TRAFFIC[tkey][1] == csrc_digest() and args.weight_decay == 0.0 \
+            and (dom == "worker_fused" or args.placement == "server"):
+        one_pass, two_pass = q.worker_pass_model()
+        units = {"worker_fused": one_pass, "absmax": two_pass if one_pass else w.n * D,
+                 "quantize": two_pass if one_pass else w.n * D}.get(dom, D)
+        traffic = NCU_TRAFFIC[tkey][0] * units
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["achieved_gbs"],
                 "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
                 "frac": kernels[dom]["frac"], "traffic": traffic,
