@@ -76,6 +76,8 @@ def parse_args():
     ap.add_argument("--kg", type=int, default=None)
     ap.add_argument("--kx", type=int, default=None)
     ap.add_argument("--single-scale", action="store_true", help="one max-abs scale per worker")
+    ap.add_argument("--scale-block-log2", type=int, default=0,
+                    help="one max-abs scale per block of 2^K elements of a tensor (0: per tensor)")
     ap.add_argument("--weight-decay", type=float, default=0.0,
                     help="lambda of the l2 term g + lambda * (held weights); 0: none")
     ap.add_argument("--e2e-steps", type=int, default=3)
@@ -96,6 +98,8 @@ def get_workload(args):
         kw["kx"] = args.kx
     if args.single_scale:
         kw["per_tensor_scale"] = False
+    if args.scale_block_log2 > 0:
+        kw["scale_block"] = 1 << args.scale_block_log2
     return w.with_(**kw) if kw else w
 
 

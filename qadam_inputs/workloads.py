@@ -32,6 +32,7 @@ class Workload:
     lr: float = 1e-3
     seed: int = 20200429
     per_tensor_scale: bool = True     # one max-abs scale per tensor (False: one per vector)
+    scale_block: int = 0              # > 0: one scale per block of this many elements of a tensor
 
     @property
     def d(self) -> int:
@@ -39,12 +40,23 @@ class Workload:
 
     @property
     def num_segments(self) -> int:
-        return len(self.seg_len) if self.per_tensor_scale else 1
+        return len(self.scale_seg_len)
 
     @property
     def scale_seg_len(self) -> Tuple[int, ...]:
-        """Segment lengths as the quantizer sees them."""
-        return self.seg_len if self.per_tensor_scale else (self.d,)
+        """Segment lengths as the quantizer sees them: the tensors (or the whole vector),
+        each cut into blocks of `scale_block` elements when that is set (the last block of
+        a tensor may be shorter)."""
+        base = self.seg_len if self.per_tensor_scale else (self.d,)
+        if self.scale_block <= 0:
+            return base
+        out = []
+        for ln in base:
+            full, rest = divmod(ln, self.scale_block)
+            out.extend([self.scale_block] * full)
+            if rest:
+                out.append(rest)
+        return tuple(out)
 
     def with_(self, **kw) -> "Workload":
         return replace(self, **kw)

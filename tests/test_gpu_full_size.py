@@ -110,6 +110,14 @@ def test_flat28_worker_count_sweep_ends_full_size():
     _run_full(qi.get_workload("flat28", n=4), qb.PLACE_WORKER, sample_e_workers=(2,))
 
 
+def test_flat28_block_scales_full_size():
+    # one scale per 2^20 elements: every (worker, block) pair fits on chip, so the whole
+    # worker side of the 2^28-element vector goes through the on-chip kernel
+    w = qi.get_workload("flat28", n=4).with_(scale_block=1 << 20)
+    _run_full(w, qb.PLACE_SERVER, sample_e_workers=(1,))
+    _run_full(w, qb.PLACE_WORKER, sample_e_workers=(3,))
+
+
 def test_bert_base_n16_full_size_both_placements():
     w = qi.get_workload("bert_base")
     _run_full(w, qb.PLACE_SERVER, sample_e_workers=(0, 9))

@@ -61,3 +61,11 @@ def test_he_init():
     x = qi.initial_weights(_small("gauss_worker", w0="he"))
     assert abs(x[:3000].std().item() / np.sqrt(2 / 27) - 1) < 0.05
     assert torch.all(x[3000:3064] == 1) and torch.all(x[3064:] == 0)
+
+
+def test_scale_blocks_cut_every_tensor():
+    w = qi.get_workload("flat20").with_(scale_block=1 << 18)
+    assert w.scale_seg_len == (1 << 18,) * 4 and w.num_segments == 4
+    r = qi.get_workload("resnet18_qg").with_(scale_block=100000)
+    assert sum(r.scale_seg_len) == r.d and max(r.scale_seg_len) == 100000
+    assert r.num_segments == sum(-(-ln // 100000) for ln in r.seg_len)
