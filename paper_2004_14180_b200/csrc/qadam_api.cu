@@ -295,13 +295,15 @@ WorkerResidentKernel pick_worker_resident(const qadam_ctx* c, bool l2) {
   }
 }
 
-// With the l2 term and the moments on the server the streaming launches run instead of the
-// on-chip kernel: its 8 load-side warps fetch the held weights from global memory with
-// nothing to hide the latency behind, and lose (measured: 6.6 ms against 2.5 + 4.5 ms for
-// everything on the BERT-base-shaped set).  With the moments on the workers the load side
-// has 16 warps and more arithmetic per element, and the on-chip kernel wins.
+// With the l2 term, the moments on the server and held weights that are not packed codes
+// of at most 8 bits, the streaming launches run instead of the on-chip kernel: its 8
+// load-side warps would fetch the held weights from global memory with nothing to hide the
+// latency behind, and lose (measured).  Packed codes of at most 8 bits are fetched a tile
+// ahead; with the moments on the workers the load side has 16 warps and more arithmetic
+// per element, and the on-chip kernel wins either way.
 bool l2_split(const qadam_ctx* c) {
-  return c->lambda != 0.0f && c->cfg.placement == QADAM_PLACE_SERVER;
+  return c->lambda != 0.0f && c->cfg.placement == QADAM_PLACE_SERVER &&
+         !(c->cfg.kx >= 0 && c->geo.xbits <= 8);
 }
 
 // grids of the split worker kernels (they depend on whether the l2 term is on)

@@ -38,6 +38,32 @@ struct WorkerParams {
   float lambda;
 };
 
+// Packed weight codes of at most 8 bits: the two 32-bit words that hold this lane's 4 codes
+// of a 128-element row (row_elem: first element of the row).  Split from the decode so
+// that a kernel can issue the loads a tile ahead of their use.
+__device__ __forceinline__ void held_fetch8(const WorkerParams& p, long long row_elem, int lane,
+                                            unsigned& lo, unsigned& hi) {
+  const unsigned* words = reinterpret_cast<const unsigned*>(p.wcodes + row_elem * p.xbits / 8);
+  const int F = 4 * p.xbits;                            // bits per lane = words per row
+  const int w = (F * lane) >> 5;
+  lo = __ldg(words + w);
+  hi = __ldg(words + (w + 1 < F ? w + 1 : w));
+}
+// ... and their values: (code - 2^kx) times the grid step, exact.
+__device__ __forceinline__ void held_decode8(const WorkerParams& p, int lane, unsigned lo, unsigned hi,
+                                             float out[4]) {
+  const int F = 4 * p.xbits;
+  const unsigned v = __funnelshift_r(lo, hi, (F * lane) & 31);
+  const unsigned f = F == 32 ? v : (v & ((1u << F) - 1u));
+  const unsigned mask = (1u << p.xbits) - 1u;
+  const float step = exp2i(-(p.kx + 1));
+  // code -> float without a conversion: 2^23 + code as a bit pattern, minus 2^23 + 2^kx
+  const float bias = -(8388608.0f + (float)(1 << p.kx));
+#pragma unroll
+  for (int c = 0; c < 4; ++c)
+    out[c] = __fmul_rn(__fadd_rn(__uint_as_float(0x4b000000u | ((f >> (c * p.xbits)) & mask)), bias), step);
+}
+
 // The weights a worker holds for this lane's 4 elements of a 128-element row: the broadcast
 // Q_x(x) decoded from its packed codes (code - 2^kx times the grid step, exact), or x itself
 // when the weights are not quantized.  row_elem: first element of the row.
@@ -48,20 +74,19 @@ __device__ __forceinline__ void held_weights4(const WorkerParams& p, long long r
     out[0] = v.x; out[1] = v.y; out[2] = v.z; out[3] = v.w;
     return;
   }
+  if (p.xbits <= 8) {
+    unsigned lo, hi;
+    held_fetch8(p, row_elem, lane, lo, hi);
+    held_decode8(p, lane, lo, hi, out);
+    return;
+  }
   const unsigned char* row = p.wcodes + row_elem * p.xbits / 8;
   const unsigned mask = (1u << p.xbits) - 1u;
   const float step = exp2i(-(p.kx + 1));
-  // code -> float without a conversion: 2^23 + code as a bit pattern, minus 2^23 + 2^kx
   const float bias = -(8388608.0f + (float)(1 << p.kx));
   auto value = [&](unsigned code) {
     return __fmul_rn(__fadd_rn(__uint_as_float(0x4b000000u | code), bias), step);
   };
-  if (p.xbits <= 8) {
-    const unsigned f = unpack_row_field(row, p.xbits, lane);          // the lane's 4 codes
-#pragma unroll
-    for (int c = 0; c < 4; ++c) out[c] = value((f >> (c * p.xbits)) & mask);
-    return;
-  }
   const unsigned* words = reinterpret_cast<const unsigned*>(row);
   const int row_words = 4 * p.xbits;                    // 128 codes
   const int half = 2 * p.xbits;                         // two codes, at most 32 bits
@@ -81,6 +106,15 @@ __device__ __forceinline__ void add_l2_term(const WorkerParams& p, long long row
                                             float gg[4]) {
   float w[4];
   held_weights4(p, row_elem, lane, w);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) gg[c] = __fadd_rn(gg[c], __fmul_rn(p.lambda, w[c]));
+}
+
+// The same from codes fetched earlier with held_fetch8.
+__device__ __forceinline__ void add_l2_term_fetched(const WorkerParams& p, int lane, unsigned lo, unsigned hi,
+                                                    float gg[4]) {
+  float w[4];
+  held_decode8(p, lane, lo, hi, w);
 #pragma unroll
   for (int c = 0; c < 4; ++c) gg[c] = __fadd_rn(gg[c], __fmul_rn(p.lambda, w[c]));
 }

@@ -308,7 +308,39 @@ worker_resident_kernel(const WorkerResidentParams rp) {
     const int row0 = tid / kRColThreads;
     int s = 0;
     unsigned ph = 0;
+    // l2 term with packed weights of at most 8 bits: the code words of a tile are fetched
+    // while the tile before it is processed (and the descriptor of the tile after it is
+    // read), so that their latency stays off the path.  hw_*: words of the tile about to be
+    // processed, one pair per row of this thread.
+    constexpr int kMineL = kRows / kLRowStep;
+    // (With the moments on the workers the 16 load-side warps hide that latency themselves,
+    // and the extra registers cost more than the fetch ahead gains: measured.)
+    const bool pref = L2 && !WM && p.kx >= 0 && p.xbits <= 8;
+    unsigned hw_lo[kMineL], hw_hi[kMineL];
+    int pj = my_tiles > 0 ? (int)((long long)cta % rp.TR) : 0;      // index of the tile whose descriptor is in `ahead`
+    RTile ahead = RTile{0, 0, 0, 0, 0};
+    auto step_j = [&]() { pj += ctas; while (pj >= rp.TR) pj -= rp.TR; };
+    auto fetch_rows = [&](const RTile& t, unsigned (&lo)[kMineL], unsigned (&hi)[kMineL]) {
+#pragma unroll
+      for (int r = 0; r < kMineL; ++r) {
+        const int q = row0 + r * kLRowStep;
+        lo[r] = hi[r] = 0u;
+        if (q * kRowElems + gt * 4 < t.count)
+          held_fetch8(p, t.off + q * kRowElems + (gt >> 5) * 128, lane, lo[r], hi[r]);
+      }
+    };
+    if (pref && my_tiles > 0) {
+      fetch_rows(rp.rtiles[pj], hw_lo, hw_hi);                       // tile 0
+      step_j();
+      if (my_tiles > 1) ahead = rp.rtiles[pj];                       // descriptor of tile 1
+    }
     for (long long i = 0; i < my_tiles; ++i) {
+      unsigned nx_lo[kMineL], nx_hi[kMineL];
+      if (pref && i + 1 < my_tiles) {
+        fetch_rows(ahead, nx_lo, nx_hi);                             // words of tile i + 1
+        step_j();
+        if (i + 2 < my_tiles) ahead = rp.rtiles[pj];                 // descriptor of tile i + 2
+      }
       if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->e_full[s], ph, abort_flag, p.status))) break;
       RLoadHeader* hdp = &ps->load_hd[i & (kRHeaders - 1)];
       const int slot = hdp->slot, count = hdp->count;
@@ -336,7 +368,10 @@ worker_resident_kernel(const WorkerResidentParams rp) {
           if (q * kRowElems + gt * 4 >= count) continue;               // warp-uniform
           float gg[4] = {g4[r].x, g4[r].y, g4[r].z, g4[r].w};
           float ee[4] = {e4[r].x, e4[r].y, e4[r].z, e4[r].w};
-          if constexpr (L2) add_l2_term(p, off + q * kRowElems + (gt >> 5) * 128, lane, gg);
+          if constexpr (L2) {
+            if (pref) add_l2_term_fetched(p, lane, hw_lo[r], hw_hi[r], gg);
+            else add_l2_term(p, off + q * kRowElems + (gt >> 5) * 128, lane, gg);
+          }
           float mm[4] = {m4[r].x, m4[r].y, m4[r].z, m4[r].w};
           float vs[4] = {v4[r].x, v4[r].y, v4[r].z, v4[r].w};
           float uu[4];
@@ -353,12 +388,16 @@ worker_resident_kernel(const WorkerResidentParams rp) {
         }
       } else {
 #pragma unroll
-        for (int q = row0; q < kRows; q += kLRowStep) {
+        for (int r = 0; r < kMineL; ++r) {
+          const int q = row0 + r * kLRowStep;
           if (q * kRowElems + gt * 4 < count) {
             const float4 g4 = *reinterpret_cast<const float4*>(su + q * kRowElems);
             const float4 e4 = *reinterpret_cast<const float4*>(se + q * kRowElems);
             float gg[4] = {g4.x, g4.y, g4.z, g4.w};
-            if constexpr (L2) add_l2_term(p, hdp->off + q * kRowElems + (gt >> 5) * 128, lane, gg);
+            if constexpr (L2) {
+              if (pref) add_l2_term_fetched(p, lane, hw_lo[r], hw_hi[r], gg);
+              else add_l2_term(p, hdp->off + q * kRowElems + (gt >> 5) * 128, lane, gg);
+            }
             const float4 u4 = make_float4(__fadd_rn(gg[0], e4.x), __fadd_rn(gg[1], e4.y), __fadd_rn(gg[2], e4.z),
                                           __fadd_rn(gg[3], e4.w));
             *reinterpret_cast<float4*>(su + q * kRowElems) = u4;
@@ -375,6 +414,10 @@ worker_resident_kernel(const WorkerResidentParams rp) {
       if (lane == 0) {
         mbar_arrive(&ps->e_empty[s]);                            // the stage has been read: it can be refilled
         mbar_arrive(&ps->hd_ready[i & (kRHeaders - 1)]);         // the header's maximum is complete
+      }
+      if constexpr (L2) {
+#pragma unroll
+        for (int r = 0; r < kMineL; ++r) { hw_lo[r] = nx_lo[r]; hw_hi[r] = nx_hi[r]; }
       }
       if (++s == estages) { s = 0; ph ^= 1u; }
     }

@@ -263,6 +263,26 @@ def test_on_chip_worker_capacity_boundary(placement):
             assert two > 0, "no pair took the streaming launches"
 
 
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+@pytest.mark.parametrize("kx", [0, 3, 6, 9, -1])
+def test_on_chip_worker_l2_term_many_tiles(kx, placement):
+    # the l2 term inside the on-chip kernel with several tiles per CTA: the held-weight
+    # codes of a tile are fetched while the tile before it is processed (widths up to 8
+    # bits); wider codes and unquantized weights are read in place or take the streaming
+    # launches
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    seg = [sms * 3 * 4096 + 300, 5000, 70000, 129]
+    n, d = 3, sum([sms * 3 * 4096 + 300, 5000, 70000, 129])
+    rng = np.random.default_rng(40 + kx)
+    x1 = (rng.standard_normal(d) * 0.3).astype(np.float32)
+    p = Pair(seg, n, 0, kx, placement, x1=x1)
+    for lam in (5e-4, 0.05, 0.0):
+        p.set_regularization(lam)
+        p.step(_rand_grads(rng, n, d))
+        p.compare_state()
+    p.close()
+
+
 # ---------------------------------------------------------------- l2 term and step-dependent rates
 
 @pytest.mark.parametrize("placement", [S_MODE, W_MODE])
