@@ -184,7 +184,6 @@ struct qadam_ctx {
   // persistent pipelined server pass (ternary codes): stages > 0 when in use
   float lambda = 0.0f;       // l2 term (qadam_set_regularization)
   int pipe_stages = 0;
-  int pipe_groups = 2;
   int pipe_skip_16ths = 2;   // zero skipping while at most this many sixteenths of the workers are live
   size_t pipe_smem = 0;
   CUtensorMap codes_map;
@@ -257,7 +256,7 @@ ServerKernel pick_server(const qadam_ctx* c) {
   }
 }
 
-using PipeKernel = void (*)(const ServerParams, const CUtensorMap, const Tile*, int, int, int, int, int);
+using PipeKernel = void (*)(const ServerParams, const CUtensorMap, const Tile*, int, int, int, int);
 
 template <bool SM, int GB>
 PipeKernel pick_pipe_n(int n) {
@@ -464,17 +463,12 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
     const size_t head = pipe_head_bytes(table);
     const char* env = std::getenv("QADAM_SERVER_KERNEL");
     const bool want_plain = env && std::strcmp(env, "plain") == 0;
-    const int fit = std::min((int)(((size_t)max_smem - head) / sb), kPipeMaxStages);
-    // three consumer groups when that still leaves a ring of six stages, else two
-    const char* genv = std::getenv("QADAM_SERVER_GROUPS");
-    int groups = genv ? std::atoi(genv) : (pipe_legal_stages(fit, 3) >= 6 ? 3 : 2);
-    groups = std::max(2, std::min(groups, kPipeMaxGroups));
-    const int stages = pipe_legal_stages(fit, groups);
+    int stages = (int)(((size_t)max_smem - head) / sb);
+    stages = pipe_legal_stages(std::min(stages, kPipeMaxStages));
     if (!want_plain && pipe_codes && cfg->n <= kPipeMaxWorkers && stages >= 2 &&
         make_codes_tensor_map(&c->codes_map, b->gcodes, (long long)c->geo.gcode_bytes, cfg->n,
                               c->geo.gbits, table)) {
       c->pipe_stages = stages;
-      c->pipe_groups = groups;
       if (const char* sk16 = std::getenv("QADAM_SKIP_16THS")) {
         const int v = std::atoi(sk16);
         if (v >= 0 && v <= 16) c->pipe_skip_16ths = v;
@@ -489,8 +483,8 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
   plan_worker_grids(c);
   c->grid_server = resident_grid(sk, c->server_smem, c->sm_count);
   c->grid_bcast = resident_grid(weight_broadcast_kernel, 0, c->sm_count);
-  // Worker side, all workers in one call.  Segments small enough to be held by the
-  // on-chip kernel (u stays in shared memory between the
+  // Worker side, moments on the server, all workers in one call.  Segments small enough
+  // for a wave of the on-chip kernel (u = g + e stays in shared memory between the
   // max-abs reduction and the quantization, so g and e are read once) go through that
   // kernel; larger segments need two passes over memory whatever is done and take the two
   // plain streaming launches, over a tile table of their own.  The on-chip kernel needs
@@ -633,7 +627,7 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
     if (!cuda_ok(e)) return QADAM_ERR_CUDA;
     c->launches += 1;
     if (!c->geo.btiles.empty()) {
-      // the segments too large for the chip: two streaming passes over their own tile table
+      // the segments too large for a wave: two streaming passes over their own tile table
       p.tiles = c->d_btiles;
       p.tiles_per_worker = (int)c->geo.btiles.size();
       p.total_tiles = (long long)worker_count * p.tiles_per_worker;
@@ -706,8 +700,8 @@ int qadam_server_step(qadam_ctx* c, int64_t step, float lr_t) {
       const int inv_exact = (n & (n - 1)) == 0 ? 1 : 0;
       const int np = (int)c->geo.ptiles.size();
       const int pgrid = std::min(c->sm_count, np);
-      pick_pipe(c)<<<pgrid, pipe_threads(c->pipe_groups), c->pipe_smem, c->stream>>>(
-          p, c->codes_map, c->d_ptiles, np, c->pipe_stages, inv_exact, c->pipe_skip_16ths, c->pipe_groups);
+      pick_pipe(c)<<<pgrid, kPipeThreads, c->pipe_smem, c->stream>>>(p, c->codes_map, c->d_ptiles, np,
+                                                                      c->pipe_stages, inv_exact, c->pipe_skip_16ths);
     } else {
       pick_server(c)<<<grid, kThreads, c->server_smem, c->stream>>>(p);
     }

@@ -4,7 +4,7 @@
 // One CTA per SM loops over 2048-element tiles.  A producer warp brings each
 // tile's inputs (x, m, v and the n workers' code runs of 512 or 768 bytes) into a ring of
 // shared-memory stages with bulk asynchronous copies that complete on an
-// mbarrier; two or three groups of eight consumer warps take alternate tiles, decode,
+// mbarrier; two groups of eight consumer warps take alternate tiles, decode,
 // average and update in place in shared memory and write the packed broadcast; a
 // storer warp sends the updated x, m, v back with bulk stores and frees the stage.  Global-memory latency is covered by
 // the copies in flight (stages x tile bytes per SM), not by occupancy, so the
@@ -22,13 +22,13 @@
 namespace qadam {
 
 constexpr int kPipeTile = 2048;                 // elements per pipeline tile
-// Consumer groups (a launch parameter, 2 or 3): group g takes tiles g, g + groups, ...  Three
-// groups keep the issue slots busier (6 instead of 4 consumer warps per scheduler) as long
-// as the ring still has about six stages; with fewer stages two groups are faster (measured).
-constexpr int kPipeMaxGroups = 3;
+#ifndef QADAM_PIPE_GROUPS
+#define QADAM_PIPE_GROUPS 2
+#endif
+constexpr int kPipeGroups = QADAM_PIPE_GROUPS;  // consumer groups; group g takes tiles g, g + groups, ...
 constexpr int kPipeGroupThreads = 256;          // 8 warps per group, 8 elements per thread and tile
-constexpr int kPipeMaxThreads = kPipeMaxGroups * kPipeGroupThreads + 64;   // + producer warp + storer warp
-__host__ __device__ constexpr int pipe_threads(int groups) { return groups * kPipeGroupThreads + 64; }
+constexpr int kPipeConsumers = kPipeGroups * kPipeGroupThreads;
+constexpr int kPipeThreads = kPipeConsumers + 64;   // + producer warp + storer warp
 constexpr int kPipeMaxWorkers = 64;
 constexpr int kPipeMaxStages = 8;
 constexpr unsigned kSpinLimit = 1u << 22;
@@ -146,14 +146,14 @@ inline bool make_codes_tensor_map(CUtensorMap* map, const void* gcodes, long lon
   return r == CUDA_SUCCESS;
 }
 
-// The ring must hold a multiple of `groups` stages.  A stage is then always served by
+// The ring must hold a multiple of kPipeGroups stages.  A stage is then always served by
 // the same consumer group, so a thread that waits on a stage's barrier for use k + 1 has
 // itself seen use k complete.  With any other count the groups would alternate on a stage,
 // and a group running ahead could ask for the parity of use k + 1 while use k is still in
 // flight, which the barrier answers with "complete" (it reports the phase before the
 // current one): the group would then work on a stage that has not been loaded.
-__host__ __device__ inline int pipe_legal_stages(int stages, int groups) {
-  return stages / groups * groups;
+__host__ __device__ inline int pipe_legal_stages(int stages) {
+  return stages / kPipeGroups * kPipeGroups;
 }
 
 struct PipeSmem {
@@ -309,10 +309,10 @@ __host__ __device__ inline size_t pipe_head_bytes(bool table_decode) {
 // GB: bits per gradient code, 2 (ternary) or 3 (five levels); 0: any grid with p.gbits
 // (3..8) bits per code, decoded through a table of the signed level values.
 template <bool SERVER_MOMENTS, int NW, int GB>
-__global__ void __launch_bounds__(kPipeMaxThreads, 1)
+__global__ void __launch_bounds__(kPipeThreads, 1)
 server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap codes_map,
                    const Tile* __restrict__ ptiles, const int num_ptiles, const int stages,
-                   const int inv_n_exact, const int skip_16ths, const int groups) {
+                   const int inv_n_exact, const int skip_16ths) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   PipeSmem* ps = reinterpret_cast<PipeSmem*>(smem_raw);
   static_assert(GB == 0 || GB == 2 || GB == 3, "code widths of the pipelined decode");
@@ -331,7 +331,7 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
 
   if constexpr (GB == 0) {
     // signed level value of every code (code = level index + L); codes past 2L never occur
-    for (int c = tid; c < 256; c += (int)blockDim.x) {
+    for (int c = tid; c < 256; c += kPipeThreads) {
       const int q = c - p.L;
       const int a = q < 0 ? -q : q;
       float lv = 0.0f;
@@ -357,7 +357,7 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
   const int my_tiles = (int)blockIdx.x < num_ptiles
                            ? (num_ptiles - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x : 0;
 
-  if (warp == groups * (kPipeGroupThreads / 32)) {
+  if (warp == kPipeConsumers / 32) {
     // ------------------------------------------------------------------ producer
     int cur_seg = -1;
     float sc0 = 0.0f, sc1 = 0.0f;                       // scales of workers lane, lane + 32
@@ -432,7 +432,7 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
         }
       }
     }
-  } else if (warp == groups * (kPipeGroupThreads / 32) + 1) {
+  } else if (warp == kPipeConsumers / 32 + 1) {
     // ------------------------------------------------------------------ storer
     int s = 0;
     unsigned ph = 0;
@@ -460,8 +460,8 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
     if (lane == 0) bulk_wait_all();               // writes are complete before the kernel ends
   } else {
     // ------------------------------------------------------------------ consumers
-    // Groups of 8 warps take alternate tiles, so that one group computes while
-    // another waits for its data or hands its tile to the storer.  In a tile a
+    // Two groups of 8 warps take alternate tiles, so that one group computes while
+    // the other waits for its data or hands its tile to the storer.  In a tile a
     // thread owns elements 4t..4t+3 of both 1024-element rows.
     const int group = tid / kPipeGroupThreads;
     const int gt = tid - group * kPipeGroupThreads;           // 0..255
@@ -489,7 +489,7 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
     int dense_tiles_left = 0;
     int dense_span = 8;
     for (int j = 0; j < my_tiles; ++j) {
-      if (j % groups == group) {
+      if (j % kPipeGroups == group) {
         // every lane waits for itself; the warp then agrees on the outcome so that it never splits
         if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->full[s], ph, abort_flag, p.status))) break;
         unsigned char* st = stage_base + (size_t)s * stage_bytes;
