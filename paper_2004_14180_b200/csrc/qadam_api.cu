@@ -483,8 +483,8 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
   plan_worker_grids(c);
   c->grid_server = resident_grid(sk, c->server_smem, c->sm_count);
   c->grid_bcast = resident_grid(weight_broadcast_kernel, 0, c->sm_count);
-  // Worker side, moments on the server, all workers in one call.  Segments small enough
-  // for a wave of the on-chip kernel (u = g + e stays in shared memory between the
+  // Worker side, all workers in one call.  Segments small enough to be held by the
+  // on-chip kernel (u stays in shared memory between the
   // max-abs reduction and the quantization, so g and e are read once) go through that
   // kernel; larger segments need two passes over memory whatever is done and take the two
   // plain streaming launches, over a tile table of their own.  The on-chip kernel needs
@@ -627,7 +627,7 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
     if (!cuda_ok(e)) return QADAM_ERR_CUDA;
     c->launches += 1;
     if (!c->geo.btiles.empty()) {
-      // the segments too large for a wave: two streaming passes over their own tile table
+      // the segments too large for the chip: two streaming passes over their own tile table
       p.tiles = c->d_btiles;
       p.tiles_per_worker = (int)c->geo.btiles.size();
       p.total_tiles = (long long)worker_count * p.tiles_per_worker;
