@@ -43,13 +43,13 @@ NCU_TRAFFIC = {
     # kernel: (bytes per unit, digest of csrc/ at capture time)
     # profiles/dram_traffic_flat28_n16_server_moments.txt: the benchmark's own workload
     # (flat28, n = 16, moments on the server), one-pass capture of the two byte counters
-    "absmax": (8.00, "67c7e2127ef56cc9"),
-    "quantize": (12.24, "67c7e2127ef56cc9"),
-    "server": (28.03, "67c7e2127ef56cc9"),
+    "absmax": (8.00, "5d466e7428edc731"),
+    "quantize": (12.24, "5d466e7428edc731"),
+    "server": (28.03, "5d466e7428edc731"),
     # profiles/worker_resident_bert_base_n4.md: the on-chip worker kernel on the BERT-base-shaped
     # set with n = 4 (a case small enough for a multi-pass capture), scaled by the pairs it takes
-    "worker_fused:server": (12.12, "67c7e2127ef56cc9"),
-    "worker_fused:worker": (28.10, "67c7e2127ef56cc9"),
+    "worker_fused:server": (12.12, "5d466e7428edc731"),
+    "worker_fused:worker": (28.10, "5d466e7428edc731"),
 }
 
 
