@@ -283,6 +283,25 @@ def test_on_chip_worker_l2_term_many_tiles(kx, placement):
     p.close()
 
 
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_streaming_launches_only(placement, monkeypatch):
+    # QADAM_WORKER_KERNEL=split (read when the context is created) sends every pair through
+    # the two streaming launches, the route that otherwise only pairs too large for the chip,
+    # partial worker ranges and some l2 cases take
+    monkeypatch.setenv("QADAM_WORKER_KERNEL", "split")
+    rng = np.random.default_rng(70 + placement)
+    seg = [9000, 64, 129, 3 * 4096 + 640, 1, 70000]
+    n, d = 4, sum([9000, 64, 129, 3 * 4096 + 640, 1, 70000])
+    x1 = (rng.standard_normal(d) * 0.2).astype(np.float32)
+    p = Pair(seg, n, 0, 1, placement, x1=x1)
+    one, two = p.gpu.worker_pass_model()
+    assert one == 0 and two == n * p.gpu.D
+    for t in range(3):
+        p.step(_rand_grads(rng, n, d))
+        p.compare_state()
+    p.close()
+
+
 # ---------------------------------------------------------------- l2 term and step-dependent rates
 
 @pytest.mark.parametrize("placement", [S_MODE, W_MODE])
