@@ -49,6 +49,9 @@ int grad_levels(int kg, int grid) {
   return kg <= 6 ? (1 << kg) : QADAM_ERR_LEVEL;
 }
 
+constexpr int kWordCtas = 256;                       // CTAs the per-pair words are sized for
+constexpr size_t kWordBudget = (size_t)32 << 20;     // bytes of workspace they may take
+
 struct Geometry {
   std::vector<int64_t> seg_len, seg_off;
   int64_t D = 0;
@@ -64,7 +67,8 @@ struct Geometry {
   std::vector<RTile> rtiles;
   std::vector<Tile> btiles;
   long long resident_elems = 0;      // padded elements of the resident segments (one vector)
-  size_t off_rtiles = 0, off_btiles = 0;
+  size_t off_rtiles = 0, off_btiles = 0, off_words = 0;
+  size_t words_bytes = 0;            // room for the per-(pair, CTA) words of the on-chip worker kernel
 };
 
 // Splits the segments into those the on-chip worker kernel can hold (at most `capacity`
@@ -76,7 +80,10 @@ void build_resident(long long capacity, Geometry* g) {
   for (const Tile& t : g->tiles) {
     if (g->seg_tiles[t.seg] <= capacity) {
       RTile r;
-      r.off = t.off; r.count = t.count; r.seg = t.seg; r.need = g->seg_tiles[t.seg]; r.pad = 0;
+      r.off = t.off; r.count = t.count; r.seg = t.seg; r.need = g->seg_tiles[t.seg];
+      // the segment's first tile: the previous entry belongs to another segment
+      r.first = (!g->rtiles.empty() && g->rtiles.back().seg == t.seg) ? g->rtiles.back().first
+                                                                      : (int)g->rtiles.size();
       g->rtiles.push_back(r);
       g->resident_elems += t.count;
     } else {
@@ -161,6 +168,14 @@ int build_geometry(const qadam_config* c, Geometry* g) {
   wo += (size_t)round_up64((int64_t)g->tiles.size() * sizeof(RTile), 256);
   g->off_btiles = wo;
   wo += (size_t)round_up64((int64_t)g->tiles.size() * sizeof(Tile), 256);
+  // one 64-bit word per (worker, segment) pair and CTA (at most kWordCtas CTAs), as long as
+  // that stays modest; beyond it the on-chip kernel falls back to one counter per pair
+  g->off_words = wo;
+  {
+    const size_t want = (size_t)c->n * c->num_segments * kWordCtas * sizeof(unsigned long long);
+    g->words_bytes = want <= kWordBudget ? want : 0;
+    wo += (size_t)round_up64((int64_t)g->words_bytes, 256);
+  }
   g->workspace_bytes = wo + 256;
   return QADAM_OK;
 }
@@ -194,6 +209,7 @@ struct qadam_ctx {
   size_t res_smem = 0;
   RTile* d_rtiles = nullptr;
   Tile* d_btiles = nullptr;
+  unsigned long long* d_words = nullptr;   // nullptr: one counter per pair instead
   // instrumentation: event pairs of the launches since the last read
   bool profiling = false;
   struct Timed { int kind; cudaEvent_t start, stop; };
@@ -433,6 +449,7 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
     c->d_done = reinterpret_cast<unsigned*>(ws + c->geo.off_done);
     c->d_rtiles = reinterpret_cast<RTile*>(ws + c->geo.off_rtiles);
     c->d_btiles = reinterpret_cast<Tile*>(ws + c->geo.off_btiles);
+    c->d_words = c->geo.words_bytes ? reinterpret_cast<unsigned long long*>(ws + c->geo.off_words) : nullptr;
   }
 
   int dev = 0;
@@ -609,8 +626,14 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
     if (!cuda_ok(cudaMemsetAsync(p.scale_bits, 0, sizeof(unsigned) * pairs, c->stream)) ||
         !cuda_ok(cudaMemsetAsync(c->d_done, 0, sizeof(unsigned) * pairs, c->stream)))
       return QADAM_ERR_CUDA;
+    const bool use_words = c->d_words != nullptr && c->grid_resident <= kWordCtas &&
+                           std::getenv("QADAM_RESIDENT_COUNTERS") == nullptr;
+    if (use_words &&
+        !cuda_ok(cudaMemsetAsync(c->d_words, 0, sizeof(unsigned long long) * pairs * c->grid_resident, c->stream)))
+      return QADAM_ERR_CUDA;
     WorkerResidentParams rp;
     rp.w = p;
+    rp.words = use_words ? c->d_words : nullptr;
     rp.rtiles = c->d_rtiles;
     rp.done = c->d_done;
     rp.TR = (int)c->geo.rtiles.size();

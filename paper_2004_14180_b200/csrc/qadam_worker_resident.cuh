@@ -51,19 +51,30 @@ __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
   return v;
 }
 
+__device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+
 // A tile of a resident segment (padded layout, one vector).
 struct __align__(8) RTile {
   long long off;   // first element
   int count;       // elements, multiple of kAlign, at most kTileElems
   int seg;         // segment
   int need;        // tiles of that segment: what the pair's counter must reach
-  int pad;
+  int first;       // index of the segment's first tile in the list of resident tiles
 };
 
 struct WorkerResidentParams {
   WorkerParams w;
   const RTile* rtiles;    // [TR]
   unsigned* done;         // [n][S] tiles counted per pair, zeroed before the launch (as are the scales)
+  unsigned long long* words;  // [n][S][gridDim.x] or nullptr: per (pair, CTA) {tiles : 32, max |u| bits : 32},
+                              // zeroed before the launch; when given, it replaces `done` and the atomics
   long long total;        // n * TR resident tiles in all
   int TR;                 // resident tiles per worker
   int slots;              // slots of the CTA's ring (a pair gives a CTA fewer tiles than this)
@@ -245,7 +256,15 @@ worker_resident_kernel(const WorkerResidentParams rp) {
         const RLoadHeader hd = ps->load_hd[hi];
         acc_max = max(acc_max, hd.max_bits);
         acc_cnt += 1;
-        if (hd.publish) {
+        if (hd.publish && rp.words != nullptr) {
+          // one word per (pair, CTA): count and maximum travel in a single plain store, so there
+          // is nothing to order across locations (the fence is for this CTA's own dispatcher,
+          // which will read u out of the slots after seeing the word)
+          __threadfence_block();
+          st_relaxed_u64(rp.words + hd.pair * ctas + cta, ((unsigned long long)acc_cnt << 32) | acc_max);
+          acc_max = 0;
+          acc_cnt = 0;
+        } else if (hd.publish) {
           // the maximum first, then (fence) the count that lets the store side of this pair go
           if (acc_max) atomicMax(p.scale_bits + hd.pair, acc_max);
           __threadfence();
@@ -262,7 +281,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
     long long ready_pair = -1;
     unsigned ready_scale = 0;
     bool ok = true;
-    if (lane == 0 && my_tiles > 0) {
+    if (my_tiles > 0) {
       long long t = cta;
       int worker = (int)(t / rp.TR);
       int j = (int)(t - (long long)worker * rp.TR);
@@ -270,31 +289,76 @@ worker_resident_kernel(const WorkerResidentParams rp) {
       for (long long i = 0; i < my_tiles; ++i) {
         const RTile cur = rp.rtiles[j];
         const long long pair = (long long)worker * p.S + cur.seg;
-        if (pair != ready_pair) {
+        if (pair != ready_pair) {                        // warp-uniform
           ok = false;
-          for (unsigned it = 0; it < kWSpinLimit; ++it) {
-            if (ld_acquire_u32(rp.done + pair) >= (unsigned)cur.need) { ok = true; break; }
-            if (*abort_flag) break;
-            __nanosleep(it < 64 ? 40 : 400);
+          if (rp.words != nullptr) {
+            // the whole warp gathers the words of the CTAs that hold tiles of the pair:
+            // CTAs (t0 + k) mod ctas, k < min(need, ctas), t0 the pair's first tile
+            const long long t0 = (long long)worker * rp.TR + cur.first;
+            const int c0 = (int)(t0 % ctas);
+            const int kmax = cur.need < ctas ? cur.need : ctas;
+            const unsigned long long* w = rp.words + pair * ctas;
+            unsigned mx = 0;
+            for (unsigned it = 0; it < kWSpinLimit; ++it) {
+              unsigned cnt = 0;
+              mx = 0;
+              for (int k = lane; k < kmax; k += 32) {
+                int c = c0 + k;
+                if (c >= ctas) c -= ctas;
+                const unsigned long long v = ld_relaxed_u64(w + c);
+                cnt += (unsigned)(v >> 32);
+                mx = max(mx, (unsigned)v);
+              }
+              cnt = __reduce_add_sync(0xffffffffu, cnt);
+              mx = __reduce_max_sync(0xffffffffu, mx);
+              if (cnt >= (unsigned)cur.need) { ok = true; break; }
+              if (*abort_flag) break;
+              __nanosleep(it < 64 ? 40 : 400);
+            }
+            __threadfence_block();                       // the words, before u is read out of the slots
+            ready_scale = mx;
+            if (ok && lane == 0 && c0 == cta) {          // the CTA of the pair's first tile reports the scale
+              p.scale_bits[pair] = mx;
+              if (mx >= 0x7f800000u) atomicOr(p.status, 1u);
+            }
+          } else {
+            if (lane == 0) {
+              for (unsigned it = 0; it < kWSpinLimit; ++it) {
+                if (ld_acquire_u32(rp.done + pair) >= (unsigned)cur.need) { ok = true; break; }
+                if (*abort_flag) break;
+                __nanosleep(it < 64 ? 40 : 400);
+              }
+              if (ok) {
+                ready_scale = __ldcg(p.scale_bits + pair);
+                if (ready_scale >= 0x7f800000u) atomicOr(p.status, 1u);
+              }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            ready_scale = __shfl_sync(0xffffffffu, ready_scale, 0);
           }
           if (!ok) {
-            if (!*abort_flag) atomicOr(p.status, 2u);
-            *abort_flag = 1;
+            if (lane == 0) {
+              if (!*abort_flag) atomicOr(p.status, 2u);
+              *abort_flag = 1;
+            }
             break;
           }
           ready_pair = pair;
-          ready_scale = __ldcg(p.scale_bits + pair);
-          if (ready_scale >= 0x7f800000u) atomicOr(p.status, 1u);
         }
-        ok = mbar_wait_bounded(&ps->cmd_empty[cs], cph ^ 1u, abort_flag, p.status);
+        if (lane == 0) {
+          ok = mbar_wait_bounded(&ps->cmd_empty[cs], cph ^ 1u, abort_flag, p.status);
+          if (ok) {
+            RCommand* cd = &ps->cmd[cs];
+            cd->off = cur.off;
+            cd->slot = slot;
+            cd->count = cur.count;
+            cd->worker = worker;
+            cd->scale_bits = ready_scale;
+            mbar_arrive(&ps->cmd_full[cs]);
+          }
+        }
+        ok = __shfl_sync(0xffffffffu, ok, 0);
         if (!ok) break;
-        RCommand* cd = &ps->cmd[cs];
-        cd->off = cur.off;
-        cd->slot = slot;
-        cd->count = cur.count;
-        cd->worker = worker;
-        cd->scale_bits = ready_scale;
-        mbar_arrive(&ps->cmd_full[cs]);
         if (++cs == kRCmds) { cs = 0; cph ^= 1u; }
         if (++slot == rp.slots) slot = 0;
         j += ctas;

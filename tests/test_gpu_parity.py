@@ -284,6 +284,17 @@ def test_on_chip_worker_l2_term_many_tiles(kx, placement):
 
 
 @pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_on_chip_worker_counter_hand_over(placement, monkeypatch):
+    # the on-chip kernel hands a pair's scale over through one word per (pair, CTA) while the
+    # workspace has room for them, else through one counter per pair; QADAM_RESIDENT_COUNTERS
+    # (read at every call) forces the second route
+    monkeypatch.setenv("QADAM_RESIDENT_COUNTERS", "1")
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    seg = [sms * 2 * 4096 + 300, 5000, 64, 70000, 129]
+    _run(seg, 3, 0, 0, placement, T=3, seed=90 + placement)
+
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
 def test_streaming_launches_only(placement, monkeypatch):
     # QADAM_WORKER_KERNEL=split (read when the context is created) sends every pair through
     # the two streaming launches, the route that otherwise only pairs too large for the chip,
