@@ -295,19 +295,24 @@ PipeKernel pick_pipe(const qadam_ctx* c) {
 
 using WorkerResidentKernel = void (*)(const WorkerResidentParams);
 
+// With the l2 term the counter hand-over runs (the words were measured slower there).
 template <int MODE>
-WorkerResidentKernel pick_worker_resident_mode(bool worker_moments, bool l2) {
-  if (worker_moments) return l2 ? worker_resident_kernel<MODE, true, true> : worker_resident_kernel<MODE, true, false>;
-  return l2 ? worker_resident_kernel<MODE, false, true> : worker_resident_kernel<MODE, false, false>;
+WorkerResidentKernel pick_worker_resident_mode(bool worker_moments, bool l2, bool words) {
+  if (l2) return worker_moments ? worker_resident_kernel<MODE, true, true, false>
+                                : worker_resident_kernel<MODE, false, true, false>;
+  if (worker_moments) return words ? worker_resident_kernel<MODE, true, false, true>
+                                   : worker_resident_kernel<MODE, true, false, false>;
+  return words ? worker_resident_kernel<MODE, false, false, true>
+               : worker_resident_kernel<MODE, false, false, false>;
 }
 
-WorkerResidentKernel pick_worker_resident(const qadam_ctx* c, bool l2) {
+WorkerResidentKernel pick_worker_resident(const qadam_ctx* c, bool l2, bool words) {
   const bool w = c->cfg.placement == QADAM_PLACE_WORKER;
   switch (c->geo.gmode) {
-    case G_TERNARY: return pick_worker_resident_mode<G_TERNARY>(w, l2);
-    case G_FIVE:    return pick_worker_resident_mode<G_FIVE>(w, l2);
-    case G_POW2:    return pick_worker_resident_mode<G_POW2>(w, l2);
-    default:        return pick_worker_resident_mode<G_UNIFORM>(w, l2);
+    case G_TERNARY: return pick_worker_resident_mode<G_TERNARY>(w, l2, words);
+    case G_FIVE:    return pick_worker_resident_mode<G_FIVE>(w, l2, words);
+    case G_POW2:    return pick_worker_resident_mode<G_POW2>(w, l2, words);
+    default:        return pick_worker_resident_mode<G_UNIFORM>(w, l2, words);
   }
 }
 
@@ -532,18 +537,15 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
         c->res_slots = slots;
         c->res_estages = estages;
         c->res_smem = resident_smem_bytes(slots, estages, wm);
-        int per_sm = 0;
-        if (!c->geo.rtiles.empty() &&
-            cuda_ok(cudaFuncSetAttribute(pick_worker_resident(c, false), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)c->res_smem)) &&
-            cuda_ok(cudaFuncSetAttribute(pick_worker_resident(c, true), cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         (int)c->res_smem)) &&
-            cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pick_worker_resident(c, false), kRThreads,
-                                                                  c->res_smem)) &&
-            per_sm >= 1 &&
-            cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pick_worker_resident(c, true), kRThreads,
-                                                                  c->res_smem)) &&
-            per_sm >= 1)
+        bool fits = !c->geo.rtiles.empty();
+        for (int variant = 0; variant < 3 && fits; ++variant) {          // plain + words, plain, l2
+          WorkerResidentKernel k = pick_worker_resident(c, variant == 2, variant == 0);
+          int per_sm = 0;
+          fits = cuda_ok(cudaFuncSetAttribute(k, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->res_smem)) &&
+                 cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, k, kRThreads, c->res_smem)) &&
+                 per_sm >= 1;
+        }
+        if (fits)
           c->grid_resident = c->sm_count;
       }
     }
@@ -626,7 +628,8 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
     if (!cuda_ok(cudaMemsetAsync(p.scale_bits, 0, sizeof(unsigned) * pairs, c->stream)) ||
         !cuda_ok(cudaMemsetAsync(c->d_done, 0, sizeof(unsigned) * pairs, c->stream)))
       return QADAM_ERR_CUDA;
-    const bool use_words = c->d_words != nullptr && c->grid_resident <= kWordCtas &&
+    const bool l2 = c->lambda != 0.0f;
+    const bool use_words = !l2 && c->d_words != nullptr && c->grid_resident <= kWordCtas &&
                            std::getenv("QADAM_RESIDENT_COUNTERS") == nullptr;
     if (use_words &&
         !cuda_ok(cudaMemsetAsync(c->d_words, 0, sizeof(unsigned long long) * pairs * c->grid_resident, c->stream)))
@@ -644,7 +647,7 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
     cudaError_t e;
     {
       LaunchTimer lt(c, QADAM_K_WORKER_FUSED);
-      e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(pick_worker_resident(c, c->lambda != 0.0f)),
+      e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(pick_worker_resident(c, l2, use_words)),
                                       dim3(c->grid_resident), dim3(kRThreads), args, c->res_smem, c->stream);
     }
     if (!cuda_ok(e)) return QADAM_ERR_CUDA;

@@ -137,8 +137,10 @@ __host__ __device__ inline size_t resident_smem_bytes(int slots, int estages, bo
 }
 
 // MODE: grid of Q_g; WM: moments on the workers; L2: the l2 term lambda * (held weights) is
-// added to g first (the held weights are decoded from the packed broadcast, or read from x).
-template <int MODE, bool WM, bool L2>
+// added to g first (the held weights are decoded from the packed broadcast, or read from x);
+// WORDS: the hand-over goes through one word per (pair, CTA) (rp.words) instead of one
+// counter per pair (rp.done) and atomics.
+template <int MODE, bool WM, bool L2, bool WORDS>
 __global__ void __launch_bounds__(kRThreads, 1)
 worker_resident_kernel(const WorkerResidentParams rp) {
   constexpr int kLWarps = resident_load_warps(WM);          // load-side consumer warps
@@ -256,7 +258,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
         const RLoadHeader hd = ps->load_hd[hi];
         acc_max = max(acc_max, hd.max_bits);
         acc_cnt += 1;
-        if (hd.publish && rp.words != nullptr) {
+        if (WORDS && hd.publish) {
           // one word per (pair, CTA): count and maximum travel in a single plain store, so there
           // is nothing to order across locations (the fence is for this CTA's own dispatcher,
           // which will read u out of the slots after seeing the word)
@@ -291,7 +293,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
         const long long pair = (long long)worker * p.S + cur.seg;
         if (pair != ready_pair) {                        // warp-uniform
           ok = false;
-          if (rp.words != nullptr) {
+          if constexpr (WORDS) {
             // the whole warp gathers the words of the CTAs that hold tiles of the pair:
             // CTAs (t0 + k) mod ctas, k < min(need, ctas), t0 the pair's first tile
             const long long t0 = (long long)worker * rp.TR + cur.first;
