@@ -43,13 +43,13 @@ NCU_TRAFFIC = {
     # kernel: (bytes per unit, digest of csrc/ at capture time)
     # profiles/dram_traffic_flat28_n16_server_moments.txt: the benchmark's own workload
     # (flat28, n = 16, moments on the server), one-pass capture of the two byte counters
-    "absmax": (8.00, "5d466e7428edc731"),
-    "quantize": (12.24, "5d466e7428edc731"),
-    "server": (28.03, "5d466e7428edc731"),
+    "absmax": (8.00, "7bed1ed2fd2fbf57"),
+    "quantize": (12.24, "7bed1ed2fd2fbf57"),
+    "server": (28.03, "7bed1ed2fd2fbf57"),
     # profiles/worker_resident_bert_base_n4.md: the on-chip worker kernel on the BERT-base-shaped
     # set with n = 4 (a case small enough for a multi-pass capture), scaled by the pairs it takes
-    "worker_fused:server": (12.12, "5d466e7428edc731"),
-    "worker_fused:worker": (28.10, "5d466e7428edc731"),
+    "worker_fused:server": (12.12, "7bed1ed2fd2fbf57"),
+    "worker_fused:worker": (28.10, "7bed1ed2fd2fbf57"),
 }
 
 
