@@ -35,22 +35,20 @@ METRIC = "qadam_ef_step_elements_per_s"
 UNIT = "elements/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM traffic per (worker, element) or per element measured with ncu
-# (dram__bytes_read.sum + dram__bytes_write.sum of one launch divided by the units
-# it processed; profiles/ holds the captures).  Valid only for the kernel sources
-# whose digest is recorded beside it.
-NCU_TRAFFIC = {
-    # kernel: (bytes per unit, digest of csrc/ at capture time)
-    # profiles/dram_traffic_flat28_n16_server_moments.txt: the benchmark's own workload
-    # (flat28, n = 16, moments on the server), one-pass capture of the two byte counters
-    "absmax": (8.00, "7bed1ed2fd2fbf57"),
-    "quantize": (12.24, "7bed1ed2fd2fbf57"),
-    "server": (28.03, "7bed1ed2fd2fbf57"),
-    # profiles/worker_resident_bert_base_n4.md: the on-chip worker kernel on the BERT-base-shaped
-    # set with n = 4 (a case small enough for a multi-pass capture), scaled by the pairs it takes
-    "worker_fused:server": (12.12, "7bed1ed2fd2fbf57"),
-    "worker_fused:worker": (28.10, "7bed1ed2fd2fbf57"),
-}
+NOMINAL_HBM_GBS = 8000.0     # the B200's HBM3e figure the 75 % target is stated against
+
+
+def ncu_traffic():
+    """DRAM bytes per unit (a (worker, element) pair for the worker kernels, an element for the
+    server pass) taken with ncu on small cases of the same kernels, with the digest of the
+    kernel sources they were taken on.  A record whose digest is not the current one is stale
+    and not used."""
+    path = os.path.join(ROOT, "profiles", "dram_traffic.json")
+    try:
+        with open(path) as f:
+            return json.load(f)
+    except Exception:
+        return {}
 
 
 def csrc_digest() -> str:
@@ -83,6 +81,9 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true",
+                    help="skip the per-configuration records (key `configs` of the line)")
+    ap.add_argument("--config-steps", type=int, default=5)
     ap.add_argument("--sample-log2", type=int, default=None,
                     help="log2 of the per-worker sample length the oracle is timed on")
     return ap.parse_args()
@@ -285,11 +286,142 @@ def job_value(d: int, n_workers: int, world: int, ms_per_step: float) -> float:
 
 # ----------------------------------------------------------------------------- the CUDA path
 
+def kernel_table(prof, w, placement_name, q, weight_decay, peak):
+    """Per kernel: launches, time, algorithmic bytes, achieved rate and its fractions."""
+    D = q.D
+    kernels = {}
+    total_ms = sum(m for m, c in prof.values()) or 1.0
+    for name, (ms, cnt) in prof.items():
+        if cnt == 0:
+            continue
+        per = ms / cnt
+        bytes_ = algorithmic_bytes(name, w, placement_name, D, q.gcode_bytes * 8 // D, q.wcode_bytes * 8 // D,
+                                   pass_model=q.worker_pass_model(), l2_term=weight_decay != 0.0)
+        gbs = bytes_ / (per * 1e-3) / 1e9
+        kernels[name] = {"launches": int(cnt), "ms_per_launch": per, "share": ms / total_ms,
+                         "algorithmic_bytes": bytes_, "achieved_gbs": gbs,
+                         "frac": gbs / peak, "frac_of_nominal": gbs / NOMINAL_HBM_GBS}
+    return kernels
+
+
+class Measured:
+    """One workload set up on the device and timed: the context stays open for the caller."""
+
+    def __init__(self, w, placement_name, weight_decay, steps, warmup, dev, world, peak, sample_clocks):
+        import torch
+        import torch.distributed as dist
+        import qadam_inputs as qi
+        import paper_2004_14180_b200 as qb
+        self.w, self.placement_name, self.weight_decay = w, placement_name, weight_decay
+        placement = qb.PLACE_SERVER if placement_name == "server" else qb.PLACE_WORKER
+        x1 = qi.initial_weights(w, dev)
+        q = qb.QAdam(w.scale_seg_len, w.n, kg=w.kg, kx=w.kx, placement=placement, beta1=w.beta1,
+                     beta2=w.beta2, eps=w.eps, lr=w.lr, x1=x1, device=dev)
+        q.set_regularization(weight_decay)
+        del x1
+        self.q, D = q, q.D
+        # one batch of gradients, resident in HBM; the same batch feeds every step
+        g = torch.zeros(w.n, D, dtype=torch.float32, device=dev)
+        for i in range(w.n):
+            gi = qi.gradients(w, 1, i, dev)
+            g[i].copy_(q.to_padded(gi))
+            del gi
+        self.g = g
+        torch.cuda.synchronize()
+
+        def sync_all():
+            torch.cuda.synchronize()
+            if world > 1:
+                dist.barrier()
+                torch.cuda.synchronize()
+        self.sync_all = sync_all
+
+        self.step = 0
+        for _ in range(max(3, warmup)):
+            self.step += 1
+            q.step(self.step, g)
+        sync_all()
+        q.profile(True)
+        q.profile_read()
+        launches0 = q.launches
+        clocks = ClockSampler(dev.index or 0) if sample_clocks else None
+        if clocks:
+            time.sleep(0.25)
+        sync_all()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            self.step += 1
+            q.step(self.step, g)
+        e1.record()
+        sync_all()
+        ms_total = e0.elapsed_time(e1)
+        self.clock_info = clocks.stop() if clocks else None
+        prof = q.profile_read()
+        q.profile(False)
+        self.gpu_launches = q.launches - launches0
+        self.status = q.poll_status()
+        self.ms_step = max_over_ranks(ms_total, world, dev) / steps
+        self.value = job_value(w.d, w.n, world, self.ms_step)
+        self.kernels = kernel_table(prof, w, placement_name, q, weight_decay, peak)
+        self.step_bytes = sum(k["algorithmic_bytes"] * k["launches"] for k in self.kernels.values()) / steps
+
+    def close(self):
+        self.q.close()
+        self.g = None
+        self.q = None
+
+
+# The configurations reported beside the headline: both large workloads over the worker-count
+# sweep, the ResNet-18-shaped sets, both placements of the moments, one run with the l2 term.
+CONFIG_RUNS = (
+    ("bert_base", None, "server", 0.0), ("bert_base", None, "worker", 0.0),
+    ("bert_base", None, "server", 5e-4),
+    ("flat28", 1, "server", 0.0), ("flat28", 4, "server", 0.0), ("flat28", 32, "server", 0.0),
+    ("flat28", 1, "worker", 0.0), ("flat28", 4, "worker", 0.0), ("flat28", 16, "worker", 0.0),
+    ("flat28", 32, "worker", 0.0),
+    ("resnet18_qg", None, "server", 0.0), ("resnet18_qg", None, "worker", 0.0),
+    ("resnet18_qg_qx_k0", None, "server", 0.0), ("resnet18_qg_qx_k0", None, "worker", 0.0),
+)
+
+
+def config_records(args, dev, world, peak):
+    """One record per configuration: step time, elements/s and every kernel's fraction of the
+    measured copy rate and of the nominal HBM rate."""
+    import torch
+    import qadam_inputs as qi
+    out = []
+    free_b, _total = torch.cuda.mem_get_info(dev)
+    for name, n, placement_name, wd in CONFIG_RUNS:
+        w = qi.get_workload(name, n=n)
+        # g, e (and the workers' m, v) dominate; skip what this device cannot hold
+        need = w.n * w.d * 4 * (4 if placement_name == "worker" else 2) + 4 * w.d * 4
+        rec = {"workload": w.name, "n_workers": w.n, "placement": placement_name, "weight_decay": wd,
+               "kg": w.kg, "kx": w.kx, "d": w.d, "segments": w.num_segments}
+        if need > 0.92 * free_b:
+            rec["skipped"] = f"needs {need >> 30} GiB of {free_b >> 30} GiB free"
+            out.append(rec)
+            continue
+        m = Measured(w, placement_name, wd, args.config_steps, 3, dev, world, peak, sample_clocks=True)
+        rec.update({"ms_per_step": m.ms_step, "value": m.value, "unit": UNIT, "steps": args.config_steps,
+                    "device_status": int(m.status), "clocks": m.clock_info,
+                    "step_frac": m.step_bytes / (m.ms_step * 1e-3) / 1e9 / peak,
+                    "step_frac_of_nominal": m.step_bytes / (m.ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+                    "l2": ("inputs larger than L2" if 8 * w.n * w.d > (1 << 28)
+                           else "fits in L2: not HBM evidence"),
+                    "kernels": {k: {"ms_per_launch": v["ms_per_launch"], "launches": v["launches"],
+                                    "achieved_gbs": v["achieved_gbs"], "frac": v["frac"],
+                                    "frac_of_nominal": v["frac_of_nominal"]} for k, v in m.kernels.items()}})
+        m.close()
+        del m
+        torch.cuda.empty_cache()
+        out.append(rec)
+    return out
+
+
 def run_b200(args):
     import torch
     import torch.distributed as dist
-    import qadam_inputs as qi
-    import paper_2004_14180_b200 as qb
 
     rank, world, local = rank_env()
     if not torch.cuda.is_available():
@@ -301,58 +433,14 @@ def run_b200(args):
         dist.init_process_group("nccl", device_id=dev)
 
     w = get_workload(args)
-    placement = qb.PLACE_SERVER if args.placement == "server" else qb.PLACE_WORKER
-    x1 = qi.initial_weights(w, dev)
-    q = qb.QAdam(w.scale_seg_len, w.n, kg=w.kg, kx=w.kx, placement=placement, beta1=w.beta1,
-                 beta2=w.beta2, eps=w.eps, lr=w.lr, x1=x1, device=dev)
-    q.set_regularization(args.weight_decay)
-    del x1
-    D = q.D
+    peak, peak_kind = measured_peak()
+    m = Measured(w, args.placement, args.weight_decay, args.steps, args.warmup, dev, world, peak,
+                 sample_clocks=True)
+    q, g, D = m.q, m.g, m.q.D
     if w.n * D * 4 <= (1 << 27):
         print(f"note: gradient input is {w.n * D * 4 >> 20} MiB, not larger than L2", file=sys.stderr)
-    # one batch of gradients, resident in HBM; the same batch feeds every step
-    g = torch.zeros(w.n, D, dtype=torch.float32, device=dev)
-    for i in range(w.n):
-        gi = qi.gradients(w, 1, i, dev)
-        g[i].copy_(q.to_padded(gi))
-        del gi
-    torch.cuda.synchronize()
-
-    def sync_all():
-        torch.cuda.synchronize()
-        if world > 1:
-            dist.barrier()
-            torch.cuda.synchronize()
-
-    step = 0
-    for _ in range(max(3, args.warmup)):
-        step += 1
-        q.step(step, g)
-    sync_all()
-
-    q.profile(True)
-    q.profile_read()
-    launches0 = q.launches
-    clocks = ClockSampler(local)
-    time.sleep(0.25)
-    sync_all()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(args.steps):
-        step += 1
-        q.step(step, g)
-    e1.record()
-    sync_all()
-    ms_total = e0.elapsed_time(e1)
-    clock_info = clocks.stop()
-    prof = q.profile_read()
-    q.profile(False)
-    gpu_launches = q.launches - launches0
-    status = q.poll_status()
-
-    ms_total = max_over_ranks(ms_total, world, dev)
-    ms_step = ms_total / args.steps
-    value = job_value(w.d, w.n, world, ms_step)
+    ms_step, value, kernels = m.ms_step, m.value, m.kernels
+    step = m.step
 
     # ---- end to end through the host-buffer entry point -------------------------------
     e2e = None
@@ -363,14 +451,14 @@ def run_b200(args):
         out_host = torch.empty(out_bytes, dtype=torch.uint8, pin_memory=True)
         step += 1
         q.step_host(step, g_host, g, out_host)          # warm-up
-        sync_all()
+        m.sync_all()
         s0, s1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         s0.record()
         for _ in range(args.e2e_steps):
             step += 1
             q.step_host(step, g_host, g, out_host)
         s1.record()
-        sync_all()
+        m.sync_all()
         ms_e2e = max_over_ranks(s0.elapsed_time(s1), world, dev) / args.e2e_steps
         e2e = {"value": job_value(w.d, w.n, world, ms_e2e), "unit": UNIT,
                "h2d_bytes_per_step": w.n * D * 4, "d2h_bytes_per_step": out_bytes,
@@ -379,32 +467,41 @@ def run_b200(args):
         del g_host, out_host
 
     # ---- roofline of the dominant kernel ---------------------------------------------
-    peak, peak_kind = measured_peak()
-    kernels = {}
-    for name, (ms, cnt) in prof.items():
-        if cnt == 0:
-            continue
-        per = ms / cnt
-        bytes_ = algorithmic_bytes(name, w, args.placement, D, q.gcode_bytes * 8 // D, q.wcode_bytes * 8 // D,
-                                   pass_model=q.worker_pass_model(), l2_term=args.weight_decay != 0.0)
-        kernels[name] = {"launches": int(cnt), "ms_per_launch": per,
-                         "share": ms / sum(m for m, c in prof.values()),
-                         "algorithmic_bytes": bytes_, "achieved_gbs": bytes_ / (per * 1e-3) / 1e9,
-                         "frac": bytes_ / (per * 1e-3) / 1e9 / peak}
     dom = max(kernels, key=lambda k: kernels[k]["launches"] * kernels[k]["ms_per_launch"])
-    traffic = None
-    tkey = f"{dom}:{args.placement}" if dom == "worker_fused" else dom
-    if tkey in NCU_TRAFFIC and NCU_TRAFFIC[tkey][1] == csrc_digest() and args.weight_decay == 0.0 \
-            and (dom == "worker_fused" or args.placement == "server"):
-        one_pass, two_pass = q.worker_pass_model()
-        units = {"worker_fused": one_pass, "absmax": two_pass if one_pass else w.n * D,
-                 "quantize": two_pass if one_pass else w.n * D}.get(dom, D)
-        traffic = NCU_TRAFFIC[tkey][0] * units
+    traffic, traffic_note = None, None
+    tkey = f"{dom}:{args.placement}"
+    trec = ncu_traffic().get(tkey)
+    if trec and args.weight_decay == 0.0:
+        if trec.get("digest") == csrc_digest():
+            one_pass, two_pass = q.worker_pass_model()
+            units = {"worker_fused": one_pass, "absmax": two_pass if one_pass else w.n * D,
+                     "quantize": two_pass if one_pass else w.n * D}.get(dom, D)
+            traffic = trec["bytes_per_unit"] * units
+            traffic_note = trec.get("case")
+        else:
+            traffic_note = "the kernel sources changed since the counters were taken"
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kernels[dom]["achieved_gbs"],
                 "peak": peak, "peak_kind": f"of {peak_kind}", "unit": "GB/s",
-                "frac": kernels[dom]["frac"], "traffic": traffic,
-                "step_frac": sum(k["algorithmic_bytes"] * k["launches"] for k in kernels.values())
-                / args.steps / (ms_step * 1e-3) / 1e9 / peak}
+                "frac": kernels[dom]["frac"], "traffic": traffic, "traffic_note": traffic_note,
+                "nominal_peak": NOMINAL_HBM_GBS, "frac_of_nominal": kernels[dom]["frac_of_nominal"],
+                "step_frac": m.step_bytes / (ms_step * 1e-3) / 1e9 / peak,
+                "step_frac_of_nominal": m.step_bytes / (ms_step * 1e-3) / 1e9 / NOMINAL_HBM_GBS,
+                # the target is stated against the nominal rate: which kernels of this run meet it
+                "target_0p75_of_nominal": {k: v["frac_of_nominal"] >= 0.75 for k, v in kernels.items()
+                                           if k != "broadcast"}}
+    sent = q.sent_bytes_per_step()
+    cfg = workload_config(w, args, extra={
+        "D_padded": D, "gcode_bits": q.gcode_bytes * 8 // D, "wcode_bits": q.wcode_bytes * 8 // D,
+        "sent_bytes_per_step": sent, "compression_ratio": q.compression_ratio(),
+        "broadcast_bytes_per_step": q.wcode_bytes})
+    clock_info, gpu_launches, status = m.clock_info, m.gpu_launches, m.status
+    m.close()
+    del m, q, g
+    torch.cuda.empty_cache()
+
+    configs = None
+    if not args.no_configs and world == 1:
+        configs = config_records(args, dev, world, peak)
 
     if rank == 0:
         cpu_baseline = None
@@ -412,22 +509,17 @@ def run_b200(args):
             sl = args.sample_log2 or 24
             v, desc, _ = time_oracle(w, args.placement, sl, steps=2, warmup=0, weight_decay=args.weight_decay)
             cpu_baseline = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle", "sample": desc}
-        sent = q.sent_bytes_per_step()
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world,
             "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step,
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "f32", "data": "synthetic",
-            "config": workload_config(w, args, extra={
-                "D_padded": D, "gcode_bits": q.gcode_bytes * 8 // D, "wcode_bits": q.wcode_bytes * 8 // D,
-                "sent_bytes_per_step": sent, "compression_ratio": q.compression_ratio(),
-                "broadcast_bytes_per_step": q.wcode_bytes}),
+            "config": cfg,
             "clocks": clock_info, "e2e": e2e, "gpu_launches": int(gpu_launches),
             "roofline": roofline, "kernels": kernels, "cpu_baseline": cpu_baseline,
-            "device_status": int(status),
+            "device_status": int(status), "configs": configs,
         }
         print(json.dumps(line), flush=True)
-    q.close()
     if world > 1:
         dist.destroy_process_group()
 

@@ -16,8 +16,13 @@
  *  - Host pointers are marked "host".
  *  - Calls enqueue work on the context's stream and return without waiting,
  *    unless stated otherwise.
- *  - Return value: QADAM_OK, or a negative qadam_error.  On an error nothing
- *    has been enqueued by that call.  Conditions found on the device (a
+ *  - Return value: QADAM_OK, or a negative qadam_error.  Arguments are checked
+ *    before anything is enqueued, so every error but QADAM_ERR_CUDA means that
+ *    the call has done nothing.  QADAM_ERR_CUDA (a CUDA call failed) may come
+ *    after clears of the scales and of the library's counters, or after the
+ *    host-to-device copy of qadam_step_host, have been enqueued; the state
+ *    buffers x, m, v, e are untouched unless a kernel was launched, and the
+ *    step counter is not advanced.  Conditions found on the device (a
  *    non-finite input, a wait that gave up) set bits of the status word.
  *  - A context is not thread-safe; distinct contexts are independent.
  *
@@ -64,7 +69,14 @@ enum { QADAM_PLACE_SERVER = 0, QADAM_PLACE_WORKER = 1 };
 /* Reading of the level set G of Section 5.1 for kg >= 2 (identical for kg = 0, 1):
  *  POW2:    {0, 2^-kg, 2^-kg+1, ..., 1}  (as printed: geometric; L = kg + 1)
  *  UNIFORM: {0, 1/2^kg, 2/2^kg, ..., 1}  (the spacing printed for X; L = 2^kg) */
-enum { QADAM_GRID_POW2 = 0, QADAM_GRID_UNIFORM = 1 };
+/*  STOCHASTIC (kg = 0 only): not a grid of Section 5.1 but the stochastic ternary operator of
+ *    the method that section compares with (TernGrad): coordinate j becomes scale * sign(u_j)
+ *    with probability |u_j| / scale and 0 otherwise (unbiased), the scale again max|u| per
+ *    (worker, segment).  The coin of padded element j of worker i at step t is word j mod 4
+ *    of the Philox4x32-10 block with counter (j/4 low, j/4 high, i, t) and key (seed low, seed
+ *    high); level 1 iff (word >> 8) * 2^-24 < fl(|u_j| / scale).  Codes, packing, the error
+ *    update and the server side are those of kg = 0. */
+enum { QADAM_GRID_POW2 = 0, QADAM_GRID_UNIFORM = 1, QADAM_GRID_STOCHASTIC = 2 };
 
 enum qadam_error {
   QADAM_OK = 0,
@@ -84,7 +96,10 @@ enum qadam_error {
 /* Bits of the device status word. */
 enum {
   QADAM_ST_NONFINITE = 1u,    /* a max-abs scale was Inf or NaN: outputs of that step are unspecified */
-  QADAM_ST_TIMEOUT = 2u       /* a bounded wait inside a kernel ran out; outputs of that step are unspecified */
+  QADAM_ST_TIMEOUT = 2u       /* a bounded wait inside a kernel ran out and the kernel returned early:
+                                 x, m, v, e and the outputs of that step are partly written and the
+                                 context cannot continue; restore the state from a copy and create a
+                                 new context */
 };
 
 typedef struct {
@@ -103,7 +118,40 @@ typedef struct {
   float eps;                  /* epsilon, > 0, added to v INSIDE the square root                 */
   float lr;                   /* default alpha, used when a step is given a negative lr_t        */
   void* stream;               /* cudaStream_t all work is enqueued on (NULL: the default stream) */
+  uint64_t seed;              /* key of the random stream; read only with QADAM_GRID_STOCHASTIC
+                                 (the quantizers of Section 5.1 are deterministic)                */
 } qadam_config;
+
+/* Which kernels a context uses where it has a choice, and two hooks for tests.  All
+ * zero (or a NULL pointer to qadam_create_ex) gives the defaults, which is what
+ * qadam_create uses.  Nothing here changes a result: every route computes the same bits.
+ *  server_kernel  AUTO: the pipelined server pass (bulk and tensor copies into shared
+ *                 memory, one CTA per SM) whenever the codes are at most 8 bits wide and
+ *                 n <= 64, else the plain grid-stride kernel.  PLAIN: always the latter.
+ *  worker_kernel  AUTO: (worker, segment) pairs that fit in the SMs' shared memory go
+ *                 through one persistent kernel that reads g and e once; larger pairs and
+ *                 calls for a part of the workers take two streaming launches (max-abs,
+ *                 then quantize).  STREAMING: always the two launches.
+ *  hand_over      how the persistent worker kernel passes a pair's scale between CTAs.
+ *                 AUTO: one 64-bit word per (pair, CTA) while those fit in 32 MB of
+ *                 workspace, else one counter per pair and atomics.  COUNTERS: always the
+ *                 latter.
+ *  wait_polls     bound on the polls of every wait inside the persistent kernels before
+ *                 the kernel gives up with QADAM_ST_TIMEOUT; 0: the default (2^22, seconds).
+ *  test_missing_tiles  TESTING ONLY.  The persistent worker kernel is told that every pair
+ *                 has this many more tiles than it has, so its waits run out: the way to
+ *                 see QADAM_ST_TIMEOUT without a fault.  Leave 0. */
+enum { QADAM_SERVER_AUTO = 0, QADAM_SERVER_PLAIN = 1 };
+enum { QADAM_WORKER_AUTO = 0, QADAM_WORKER_STREAMING = 1 };
+enum { QADAM_HANDOVER_AUTO = 0, QADAM_HANDOVER_COUNTERS = 1 };
+typedef struct {
+  int32_t server_kernel;      /* QADAM_SERVER_*   */
+  int32_t worker_kernel;      /* QADAM_WORKER_*   */
+  int32_t hand_over;          /* QADAM_HANDOVER_* */
+  uint32_t wait_polls;
+  int32_t test_missing_tiles;
+  int32_t reserved[3];        /* must be 0 */
+} qadam_options;
 
 typedef struct {
   float* x;                   /* [D] master copy x_t, updated in place                            */
@@ -139,6 +187,11 @@ int qadam_weight_code_bits(int32_t kx);
  * Q_x(x_1) into wcodes (and wresid), the first line of Algorithm 2's loop. */
 int qadam_create(const qadam_config* cfg, const qadam_buffers* bufs, qadam_ctx** out);
 
+/* The same with explicit options (host, may be NULL).  QADAM_ERR_SIZE for an unknown
+ * enumerator or a non-zero reserved field. */
+int qadam_create_ex(const qadam_config* cfg, const qadam_buffers* bufs, const qadam_options* opt,
+                    qadam_ctx** out);
+
 /* Worker side of step `step` (1-based) for workers [worker_begin, worker_begin +
  * worker_count): Algorithm 3, lines from "v = ..." to the error update.
  *   g: [worker_count][D] stochastic gradients of those workers (padded layout).
@@ -161,6 +214,37 @@ int qadam_worker_compress(qadam_ctx* ctx, int64_t step, const float* g,
  * 2^-(kx+1) on [-1/2, 1/2], clipped, ties toward zero) and wresid <- x - Q_x(x).
  * Requires that all n workers were compressed for `step`. */
 int qadam_server_step(qadam_ctx* ctx, int64_t step, float lr_t);
+
+/* The server side of step `step` for a part of the vector: Algorithm 2 when the server
+ * is sharded, each shard owning a contiguous range of x (and of m, v under
+ * PLACE_SERVER) and receiving, from every worker, the codes of that range ("Gathering
+ * all updates").  Elements [elem_begin, elem_end) of the padded layout are served
+ * exactly as qadam_server_step serves them: the same sums in the same order, the same
+ * bits in x, m, v, wcodes and wresid on that range; nothing outside it is read or
+ * written (gcodes: bytes [elem_begin*b_g/8, elem_end*b_g/8) of each worker's stream, and
+ * every worker's scales).  Both ends must be shard cuts (qadam_shard_cuts), else
+ * QADAM_ERR_SIZE.  The caller vouches that all n workers' codes of the range and all
+ * scales are in gcodes / scales (compressed here or received from elsewhere): the check of
+ * qadam_server_step on the workers compressed by THIS context does not apply.
+ * A step served by ranges stays open until qadam_finish_step; ranges of one step must not
+ * overlap (not checked: a range served twice is updated twice). */
+int qadam_server_step_range(qadam_ctx* ctx, int64_t step, float lr_t, int64_t elem_begin,
+                            int64_t elem_end);
+
+/* Closes a step that was served through qadam_server_step_range (here for some ranges,
+ * by other processes for the rest): the next worker and server calls expect step + 1.
+ * Host call, nothing is enqueued.  QADAM_ERR_STEP unless `step` is the open step. */
+int qadam_finish_step(qadam_ctx* ctx, int64_t step);
+
+/* Cuts of the padded vector into `shards` contiguous ranges of nearly equal length for a
+ * sharded server: cuts[0] = 0 <= cuts[1] <= ... <= cuts[shards] = D (host array of
+ * shards + 1 entries).  Every cut falls on a boundary of the 4096-element tiles the
+ * kernels walk (tiles never straddle a segment), so a range is a whole number of tiles
+ * and its code bytes are 16-byte aligned in every stream.  With more shards than tiles
+ * some ranges are empty.  A function of the configuration only (host call, no device
+ * needed): every process of a sharded run computes the same cuts.  QADAM_ERR_SIZE for
+ * shards < 1. */
+int qadam_shard_cuts(const qadam_config* cfg, int32_t shards, int64_t* cuts);
 
 /* One whole step from HOST memory, for callers whose gradients live on the host:
  * copies g_host ([n][D], host, ideally pinned) into g_stage (device, [n][D],
@@ -201,7 +285,8 @@ int qadam_set_regularization(qadam_ctx* ctx, float lambda);
  * The kernel's scratch (tile table, running maxima) is a fixed 260 KiB array inside
  * the library image, held by every GPU that loads the library until the process
  * ends.  Limits: D <= QADAM_STATIC_MAX_ELEMENTS and n <= QADAM_STATIC_MAX_WORKERS,
- * else QADAM_ERR_CAPACITY and nothing is enqueued.  The call allocates and frees
+ * else QADAM_ERR_CAPACITY and nothing is enqueued.  There is no status word here: a
+ * non-finite input shows only as an Inf or NaN scale.  The call allocates and frees
  * nothing.  The first call on each device looks the array's address up; make that
  * first call outside any stream capture.  All calls on a device share the one
  * array (each call rewrites and clears what it uses), so two calls that may overlap

@@ -26,6 +26,7 @@ PLACE_SERVER = 0
 PLACE_WORKER = 1
 GRID_POW2 = 0
 GRID_UNIFORM = 1
+GRID_STOCHASTIC = 2     # kg = 0 only: the stochastic ternary operator (Philox4x32-10 coins)
 ALIGN = 128
 
 
@@ -46,7 +47,7 @@ class _Problem(C.Structure):
         ("seg_len", C.POINTER(C.c_int64)), ("seg_off", C.POINTER(C.c_int64)),
         ("kg", C.c_int32), ("kx", C.c_int32), ("grid_g", C.c_int32), ("placement", C.c_int32),
         ("beta", C.c_float), ("theta", C.c_float), ("eps", C.c_float),
-        ("weight_decay", C.c_float),
+        ("weight_decay", C.c_float), ("seed", C.c_uint64),
     ]
 
 
@@ -82,7 +83,13 @@ def lib():
         L.qo_unpack_bits.restype = None
         L.qo_unpack_bits.argtypes = [u8p, C.c_int64, C.c_int32, u32p]
         L.qo_worker_step.restype = C.c_int32
-        L.qo_worker_step.argtypes = [pp, f32p, f32p, f32p, f32p, f32p, C.c_float, f32p, u8p]
+        L.qo_worker_step.argtypes = [pp, f32p, f32p, f32p, f32p, f32p, C.c_float, f32p, u8p,
+                                     C.c_int32, C.c_int64]
+        L.qo_philox4x32_10.restype = None
+        L.qo_philox4x32_10.argtypes = [u32p, u32p, u32p]
+        L.qo_quantize_grad_segment_stochastic.restype = C.c_int32
+        L.qo_quantize_grad_segment_stochastic.argtypes = [f32p, C.c_int64, C.c_int64, C.c_uint64, C.c_uint32,
+                                                          C.c_uint32, f32p, i32p, f32p]
         L.qo_broadcast_weights.restype = C.c_int32
         L.qo_broadcast_weights.argtypes = [pp, f32p, u8p, f32p]
         L.qo_server_step.restype = C.c_int32
@@ -139,6 +146,26 @@ def quantize_grad_segment(u: np.ndarray, kg: int, grid: int = GRID_POW2):
     return float(s[0]), q, r
 
 
+def philox4x32_10(ctr, key) -> np.ndarray:
+    """One block of Philox4x32-10: ctr four and key two 32-bit words -> four words."""
+    c = np.ascontiguousarray(ctr, dtype=np.uint32)
+    k = np.ascontiguousarray(key, dtype=np.uint32)
+    out = np.zeros(4, dtype=np.uint32)
+    lib().qo_philox4x32_10(_p(c, C.c_uint32), _p(k, C.c_uint32), _p(out, C.c_uint32))
+    return out
+
+
+def quantize_grad_segment_stochastic(u: np.ndarray, first_elem: int, seed: int, step: int, worker: int):
+    """Stochastic ternary operator on one segment -> (scale, q[int32], resid[float32])."""
+    u = np.ascontiguousarray(u, dtype=np.float32)
+    q = np.zeros(u.size, dtype=np.int32)
+    r = np.zeros(u.size, dtype=np.float32)
+    s = np.zeros(1, dtype=np.float32)
+    lib().qo_quantize_grad_segment_stochastic(_p(u, C.c_float), u.size, first_elem, seed, step, worker,
+                                              _p(s, C.c_float), _p(q, C.c_int32), _p(r, C.c_float))
+    return float(s[0]), q, r
+
+
 def quantize_weights(x: np.ndarray, kx: int):
     """-> (q[int32], xhat[float32], resid[float32])."""
     x = np.ascontiguousarray(x, dtype=np.float32)
@@ -178,7 +205,7 @@ class OracleState:
 
     def __init__(self, seg_len: Sequence[int], n: int, kg: int, kx: int, placement: int,
                  beta1: float, beta2: float, eps: float, grid_g: int = GRID_POW2,
-                 want_wresid: bool = False):
+                 want_wresid: bool = False, seed: int = 0):
         self.seg_len = np.ascontiguousarray(seg_len, dtype=np.int64)
         self.seg_off, self.D = layout(self.seg_len)
         self.d = int(self.seg_len.sum())
@@ -186,7 +213,8 @@ class OracleState:
         self.kg, self.kx, self.grid_g, self.placement = kg, kx, grid_g, placement
         self._prob = _Problem(self.d, self.D, self.n, self.S,
                               _p(self.seg_len, C.c_int64), _p(self.seg_off, C.c_int64),
-                              kg, kx, grid_g, placement, beta1, beta2, eps, 0.0)
+                              kg, kx, grid_g, placement, beta1, beta2, eps, 0.0, seed)
+        self.step_no = 0                  # completed steps; the next worker step is step_no + 1
         self.gcode_bytes = int(lib().qo_gcode_bytes(C.byref(self._prob)))
         self.wcode_bytes = int(lib().qo_wcode_bytes(C.byref(self._prob)))
         D = self.D
@@ -237,7 +265,6 @@ class OracleState:
     def set_regularization(self, weight_decay: float) -> None:
         """lambda of the l2 term (Section 5.1) for the steps that follow."""
         self._prob.weight_decay = weight_decay
-        self._xhat = None
 
     def held_weights(self) -> np.ndarray:
         """What the workers hold during a step: the decoded broadcast, or x itself
@@ -256,7 +283,7 @@ class OracleState:
             _p(self.m[i], C.c_float) if wm else None,
             _p(self.v[i], C.c_float) if wm else None,
             _p(self.e[i], C.c_float), lr,
-            _p(self.scales[i], C.c_float), _p(self.gcodes[i], C.c_uint8))
+            _p(self.scales[i], C.c_float), _p(self.gcodes[i], C.c_uint8), i, self.step_no + 1)
         if rc != 0:
             raise RuntimeError(f"qo_worker_step failed: {rc}")
 
@@ -283,6 +310,7 @@ class OracleState:
             _p(self.wresid, C.c_float))
         if rc != 0:
             raise RuntimeError(f"qo_server_step failed: {rc}")
+        self.step_no += 1
 
     def step(self, g_padded: np.ndarray, lr: float, threads: int = 1) -> None:
         self.workers_step(g_padded, lr, threads)

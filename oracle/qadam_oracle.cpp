@@ -60,6 +60,10 @@ int bits_for(int num_codes) {
 }
 
 bool make_grad_levels(int kg, int grid, GradLevels* out) {
+  if (grid == 2) {                        // stochastic ternary: the level set {0, 1}, kg = 0 only
+    if (kg != 0) return false;
+    grid = 0;
+  }
   if (kg < 0 || kg > 14 || (grid != 0 && grid != 1)) return false;
   GradLevels g;
   if (grid == 1) {
@@ -122,6 +126,77 @@ float dequantize_grad(int32_t qv, float s, const GradLevels& G) {
   if (qv < 0) deq = -deq;
   if (qv == 0) deq = 0.0f;
   return deq;
+}
+
+// ---------------------------------------------------------------------------
+// Philox4x32-10, the counter-based generator of Salmon, Moraes, Dror and Shaw
+// ("Parallel random numbers: as easy as 1, 2, 3", SC 2011), written from its
+// published definition: a 128-bit counter (four 32-bit words) and a 64-bit key
+// (two words) go through ten rounds; a round multiplies words 0 and 2 by two fixed
+// odd constants, keeps both halves of the 64-bit products and mixes in the other
+// two words and the key; between rounds the key words grow by two Weyl constants
+// (the golden ratio and sqrt(3) - 1 in 32-bit fixed point).
+// It is the only source of randomness anywhere in this file and is used only by the
+// stochastic ternary operator below.
+// ---------------------------------------------------------------------------
+void philox4x32_10(const uint32_t ctr[4], const uint32_t key[2], uint32_t out[4]) {
+  const uint64_t M0 = 0xD2511F53u, M1 = 0xCD9E8D57u;
+  const uint32_t W0 = 0x9E3779B9u, W1 = 0xBB67AE85u;
+  uint32_t c0 = ctr[0], c1 = ctr[1], c2 = ctr[2], c3 = ctr[3];
+  uint32_t k0 = key[0], k1 = key[1];
+  for (int round = 0; round < 10; ++round) {
+    const uint64_t p0 = M0 * (uint64_t)c0;
+    const uint64_t p1 = M1 * (uint64_t)c2;
+    const uint32_t n0 = (uint32_t)(p1 >> 32) ^ c1 ^ k0;
+    const uint32_t n1 = (uint32_t)p1;
+    const uint32_t n2 = (uint32_t)(p0 >> 32) ^ c3 ^ k1;
+    const uint32_t n3 = (uint32_t)p0;
+    c0 = n0; c1 = n1; c2 = n2; c3 = n3;
+    k0 += W0;
+    k1 += W1;
+  }
+  out[0] = c0; out[1] = c1; out[2] = c2; out[3] = c3;
+}
+
+// ---------------------------------------------------------------------------
+// The stochastic ternary operator of the method Section 5.1 compares with
+// (TernGrad): with s = |u|_inf, coordinate j becomes s * sign(u_j) with probability
+// |u_j| / s and 0 otherwise, which makes the operator unbiased, E Q(u) = u.
+// READING (how the coin is tossed): y = |u_j| / s in binary32; the coin is the top
+// 24 bits of one Philox word read as r = bits * 2^-24 in [0, 1); the level is 1 iff
+// r < y.  So the arg-max (y = 1) is always kept and a zero is never raised.
+// READING (which word): element j of the padded layout takes word j mod 4 of the
+// block with counter (low and high half of j / 4, worker, step) and key (low and
+// high half of the seed): any element of any worker at any step can be drawn alone.
+// ---------------------------------------------------------------------------
+void quantize_grad_segment_stochastic(const float* u, int64_t len, int64_t first_elem,
+                                      uint64_t seed, uint32_t step, uint32_t worker,
+                                      float* scale_out, int32_t* q, float* resid) {
+  float s = 0.0f;
+  for (int64_t j = 0; j < len; ++j) {
+    float a = std::fabs(u[j]);
+    if (a > s) s = a;
+  }
+  *scale_out = s;
+  const uint32_t key[2] = {(uint32_t)seed, (uint32_t)(seed >> 32)};
+  for (int64_t j = 0; j < len; ++j) {
+    int c = 0;
+    if (s > 0.0f) {
+      const int64_t elem = first_elem + j;
+      const uint64_t block = (uint64_t)elem >> 2;
+      const uint32_t ctr[4] = {(uint32_t)block, (uint32_t)(block >> 32), worker, step};
+      uint32_t words[4];
+      philox4x32_10(ctr, key, words);
+      const float r = (float)(words[elem & 3] >> 8) * 5.9604644775390625e-08f;   // 2^-24, exact
+      const float y = std::fabs(u[j]) / s;
+      c = (r < y) ? 1 : 0;
+    }
+    float deq = (c != 0) ? s : 0.0f;
+    if (u[j] < 0.0f) { deq = -deq; c = -c; }
+    if (c == 0) deq = 0.0f;
+    q[j] = c;
+    resid[j] = u[j] - deq;
+  }
 }
 
 // ---------------------------------------------------------------------------
@@ -232,11 +307,12 @@ typedef struct {
   const int64_t* seg_off;    // [S] padded start offsets
   int32_t kg;                // -1: Q_g = identity
   int32_t kx;                // -1: Q_x = identity (nothing broadcast in packed form)
-  int32_t grid_g;            // 0 POW2, 1 UNIFORM
+  int32_t grid_g;            // 0 POW2, 1 UNIFORM, 2 STOCHASTIC (kg = 0 only: the stochastic ternary operator)
   int32_t placement;         // where m, v live
   float beta, theta, eps;    // beta_t, theta_t of the step at hand (the caller may change them
                              // between steps: Assumption 2's theta_t = 1 - theta/t)
   float weight_decay;        // lambda of the l2 term (Section 5.1); 0: none
+  uint64_t seed;             // key of the random stream (stochastic operator only)
 } qo_problem;
 
 // Padded layout: segment s starts at the next multiple of 128 elements.
@@ -310,8 +386,22 @@ void qo_unpack_bits(const uint8_t* in, int64_t count, int32_t bits, uint32_t* co
 //   contrasts with): u = g + e, moments are the server's.
 // READING (identity Q_g): the stream is the raw binary32 of u, scale 1, e = 0.
 // ---------------------------------------------------------------------------
+void qo_philox4x32_10(const uint32_t* ctr, const uint32_t* key, uint32_t* out) {
+  philox4x32_10(ctr, key, out);
+}
+
+int32_t qo_quantize_grad_segment_stochastic(const float* u, int64_t len, int64_t first_elem,
+                                            uint64_t seed, uint32_t step, uint32_t worker,
+                                            float* scale_out, int32_t* q, float* resid) {
+  quantize_grad_segment_stochastic(u, len, first_elem, seed, step, worker, scale_out, q, resid);
+  return 0;
+}
+
+// worker, step: this worker's index and the step number (1-based); they only select the
+// random stream of the stochastic operator.
 int32_t qo_worker_step(const qo_problem* p, const float* g, const float* xhat, float* m, float* v,
-                       float* e, float alpha, float* scales, uint8_t* codes) {
+                       float* e, float alpha, float* scales, uint8_t* codes,
+                       int32_t worker, int64_t step) {
   const Hyper h = make_hyper(p->beta, p->theta, p->eps);
   GradLevels G;
   if (p->kg >= 0 && !make_grad_levels(p->kg, p->grid_g, &G)) return -1;
@@ -351,7 +441,11 @@ int32_t qo_worker_step(const qo_problem* p, const float* g, const float* xhat, f
       continue;
     }
     q.assign((size_t)len, 0);
-    quantize_grad_segment(u.data(), len, G, &scales[s], q.data(), e + off);
+    if (p->grid_g == 2)
+      quantize_grad_segment_stochastic(u.data(), len, off, p->seed, (uint32_t)step, (uint32_t)worker,
+                                       &scales[s], q.data(), e + off);
+    else
+      quantize_grad_segment(u.data(), len, G, &scales[s], q.data(), e + off);
     code.assign((size_t)plen, (uint32_t)G.L);            // pads: level 0
     for (int64_t j = 0; j < len; ++j) code[j] = (uint32_t)(q[j] + G.L);
     pack_bits(code.data(), plen, G.bits, codes + off * G.bits / 8);

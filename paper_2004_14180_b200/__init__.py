@@ -7,9 +7,11 @@ memory and streams.  There is no CPU fallback: importing the binding without
 the built library, or calling it without a CUDA device, raises.
 """
 from .binding import (  # noqa: F401
-    PLACE_SERVER, PLACE_WORKER, GRID_POW2, GRID_UNIFORM,
+    PLACE_SERVER, PLACE_WORKER, GRID_POW2, GRID_UNIFORM, GRID_STOCHASTIC,
     ST_NONFINITE, ST_TIMEOUT,
-    QAdamError, QAdamConfig, QAdamBuffers, QAdam,
+    QAdamError, QAdamConfig, QAdamBuffers, QAdamOptions, QAdam,
+    SERVER_AUTO, SERVER_PLAIN, WORKER_AUTO, WORKER_STREAMING, HANDOVER_AUTO, HANDOVER_COUNTERS,
+    qadam_create_ex, qadam_server_step_range, qadam_finish_step, qadam_shard_cuts,
     library_path, load_library, exported_symbols,
     qadam_query_sizes, qadam_grad_code_bits, qadam_weight_code_bits,
     qadam_create, qadam_worker_compress, qadam_server_step, qadam_step_host,

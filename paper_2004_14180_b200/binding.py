@@ -13,7 +13,7 @@ from typing import Optional, Sequence
 import torch
 
 PLACE_SERVER, PLACE_WORKER = 0, 1
-GRID_POW2, GRID_UNIFORM = 0, 1
+GRID_POW2, GRID_UNIFORM, GRID_STOCHASTIC = 0, 1, 2
 ST_NONFINITE, ST_TIMEOUT = 1, 2
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -25,7 +25,12 @@ exported_symbols = (
     "qadam_launch_count", "qadam_destroy", "qadam_strerror", "qadam_last_cuda_error",
     "qadam_profile_enable", "qadam_profile_read", "qadam_worker_scales_static",
     "qadam_worker_pass_model", "qadam_set_moment_rates", "qadam_set_regularization",
+    "qadam_create_ex", "qadam_server_step_range", "qadam_finish_step", "qadam_shard_cuts",
 )
+
+SERVER_AUTO, SERVER_PLAIN = 0, 1
+WORKER_AUTO, WORKER_STREAMING = 0, 1
+HANDOVER_AUTO, HANDOVER_COUNTERS = 0, 1
 
 STATIC_MAX_ELEMENTS = 1 << 26
 STATIC_MAX_WORKERS = 1024
@@ -48,7 +53,14 @@ class QAdamConfig(C.Structure):
         ("seg_len", C.POINTER(C.c_int64)),
         ("kg", C.c_int32), ("kx", C.c_int32), ("grid_g", C.c_int32), ("placement", C.c_int32),
         ("beta1", C.c_float), ("beta2", C.c_float), ("eps", C.c_float), ("lr", C.c_float),
-        ("stream", C.c_void_p),
+        ("stream", C.c_void_p), ("seed", C.c_uint64),
+    ]
+
+
+class QAdamOptions(C.Structure):
+    _fields_ = [
+        ("server_kernel", C.c_int32), ("worker_kernel", C.c_int32), ("hand_over", C.c_int32),
+        ("wait_polls", C.c_uint32), ("test_missing_tiles", C.c_int32), ("reserved", C.c_int32 * 3),
     ]
 
 
@@ -88,6 +100,14 @@ def load_library():
     L.qadam_weight_code_bits.argtypes = [C.c_int32]
     L.qadam_create.restype = C.c_int
     L.qadam_create.argtypes = [cfgp, bufp, C.POINTER(C.c_void_p)]
+    L.qadam_create_ex.restype = C.c_int
+    L.qadam_create_ex.argtypes = [cfgp, bufp, C.POINTER(QAdamOptions), C.POINTER(C.c_void_p)]
+    L.qadam_server_step_range.restype = C.c_int
+    L.qadam_server_step_range.argtypes = [C.c_void_p, C.c_int64, C.c_float, C.c_int64, C.c_int64]
+    L.qadam_finish_step.restype = C.c_int
+    L.qadam_finish_step.argtypes = [C.c_void_p, C.c_int64]
+    L.qadam_shard_cuts.restype = C.c_int
+    L.qadam_shard_cuts.argtypes = [cfgp, C.c_int32, C.POINTER(C.c_int64)]
     L.qadam_worker_compress.restype = C.c_int
     L.qadam_worker_compress.argtypes = [C.c_void_p, C.c_int64, C.c_void_p, C.c_int32, C.c_int32, C.c_float]
     L.qadam_server_step.restype = C.c_int
@@ -155,6 +175,30 @@ def qadam_create(cfg: QAdamConfig, bufs: QAdamBuffers) -> int:
     ctx = C.c_void_p()
     _check(load_library().qadam_create(C.byref(cfg), C.byref(bufs), C.byref(ctx)), "qadam_create")
     return ctx.value
+
+
+def qadam_create_ex(cfg: QAdamConfig, bufs: QAdamBuffers, opt: Optional[QAdamOptions]) -> int:
+    ctx = C.c_void_p()
+    _check(load_library().qadam_create_ex(C.byref(cfg), C.byref(bufs),
+                                          C.byref(opt) if opt is not None else None, C.byref(ctx)),
+           "qadam_create_ex")
+    return ctx.value
+
+
+def qadam_server_step_range(ctx: int, step: int, lr_t: float, elem_begin: int, elem_end: int) -> None:
+    _check(load_library().qadam_server_step_range(ctx, step, lr_t, elem_begin, elem_end),
+           "qadam_server_step_range")
+
+
+def qadam_finish_step(ctx: int, step: int) -> None:
+    _check(load_library().qadam_finish_step(ctx, step), "qadam_finish_step")
+
+
+def qadam_shard_cuts(cfg: QAdamConfig, shards: int):
+    """-> shards + 1 element offsets, the ranges a sharded server may be cut into (host only)."""
+    cuts = (C.c_int64 * (max(0, shards) + 1))()
+    _check(load_library().qadam_shard_cuts(C.byref(cfg), shards, cuts), "qadam_shard_cuts")
+    return list(cuts)
 
 
 def qadam_worker_compress(ctx: int, step: int, g_ptr: int, worker_begin: int, worker_count: int,
@@ -235,7 +279,8 @@ class QAdam:
                  placement: int = PLACE_SERVER, beta1: float = 0.9, beta2: float = 0.999,
                  eps: float = 1e-8, lr: float = 1e-3, grid_g: int = GRID_POW2,
                  x1: Optional[torch.Tensor] = None, want_wresid: bool = False,
-                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None):
+                 device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None,
+                 seed: int = 0, options: Optional[QAdamOptions] = None):
         load_library()
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2004_14180_b200 needs a CUDA device; there is no CPU path")
@@ -248,7 +293,7 @@ class QAdam:
             d=sum(self.seg_len), n=self.n, num_segments=len(self.seg_len), seg_len=self._seg_arr,
             kg=kg, kx=kx, grid_g=grid_g, placement=placement, beta1=beta1, beta2=beta2, eps=eps,
             lr=lr, stream=(stream.cuda_stream if stream is not None else
-                           torch.cuda.current_stream(self.device).cuda_stream))
+                           torch.cuda.current_stream(self.device).cuda_stream), seed=seed)
         sz = qadam_query_sizes(self.cfg)
         self.d, self.D, self.S = sum(self.seg_len), sz["D"], len(self.seg_len)
         self.seg_off = sz["seg_off"]
@@ -278,7 +323,8 @@ class QAdam:
                 status=self.status.data_ptr())
             # buffers were filled on torch's current stream; the context may use another
             torch.cuda.current_stream(self.device).synchronize()
-            self.ctx = qadam_create(self.cfg, self.bufs)
+            self.ctx = (qadam_create(self.cfg, self.bufs) if options is None
+                        else qadam_create_ex(self.cfg, self.bufs, options))
 
     # layout -------------------------------------------------------------------
     def to_padded(self, logical: torch.Tensor) -> torch.Tensor:
@@ -313,6 +359,15 @@ class QAdam:
 
     def server_step(self, step: int, lr: float = -1.0) -> None:
         qadam_server_step(self.ctx, step, lr)
+
+    def server_step_range(self, step: int, elem_begin: int, elem_end: int, lr: float = -1.0) -> None:
+        qadam_server_step_range(self.ctx, step, lr, elem_begin, elem_end)
+
+    def finish_step(self, step: int) -> None:
+        qadam_finish_step(self.ctx, step)
+
+    def shard_cuts(self, shards: int):
+        return qadam_shard_cuts(self.cfg, shards)
 
     def step(self, step: int, g: torch.Tensor, lr: float = -1.0) -> None:
         self.worker_compress(step, g, 0, self.n, lr)

@@ -12,7 +12,7 @@ LIB = os.path.join(_HERE, "libqadam.so")
 SOURCES = [os.path.join(CSRC, "qadam_api.cu"), os.path.join(CSRC, "qadam_noalloc.cu")]
 HEADERS = [os.path.join(CSRC, "qadam_device.cuh"), os.path.join(CSRC, "qadam_kernels.cuh"),
            os.path.join(CSRC, "qadam_server_pipe.cuh"),
-           os.path.join(CSRC, "qadam_worker_resident.cuh"),
+           os.path.join(CSRC, "qadam_worker_resident.cuh"), os.path.join(CSRC, "qadam_host.h"),
            os.path.join(_ROOT, "include", "qadam.h")]
 
 NVCC_FLAGS = [

@@ -11,11 +11,10 @@
 #include <new>
 #include <vector>
 
+#include "qadam_host.h"
 #include "qadam_kernels.cuh"
 #include "qadam_server_pipe.cuh"
 #include "qadam_worker_resident.cuh"
-
-#include <cstdlib>
 
 using namespace qadam;
 
@@ -31,6 +30,12 @@ inline bool cuda_ok(cudaError_t e) {
   return true;
 }
 
+}  // namespace
+
+void qadam::record_cuda_error(int cuda_error) { g_last_cuda_error = cuda_error; }
+
+namespace {
+
 inline int64_t round_up64(int64_t v, int64_t a) { return (v + a - 1) / a * a; }
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
@@ -42,6 +47,7 @@ int bits_for(int num_codes) {
 
 // Positive levels L of G for (kg, grid), or a negative error.
 int grad_levels(int kg, int grid) {
+  if (grid == QADAM_GRID_STOCHASTIC) return kg == 0 ? 1 : QADAM_ERR_LEVEL;
   if (grid != QADAM_GRID_POW2 && grid != QADAM_GRID_UNIFORM) return QADAM_ERR_LEVEL;
   if (kg < 0) return QADAM_ERR_LEVEL;
   if (kg <= 1) return kg + 1;                          // both grids: {0,1}, {0,1/2,1}
@@ -73,14 +79,14 @@ struct Geometry {
 
 // Splits the segments into those the on-chip worker kernel can hold (at most `capacity`
 // tiles per (worker, segment) pair) and the rest, each with a tile table of its own.
-void build_resident(long long capacity, Geometry* g) {
+void build_resident(long long capacity, int missing_tiles, Geometry* g) {
   g->rtiles.clear();
   g->btiles.clear();
   g->resident_elems = 0;
   for (const Tile& t : g->tiles) {
     if (g->seg_tiles[t.seg] <= capacity) {
       RTile r;
-      r.off = t.off; r.count = t.count; r.seg = t.seg; r.need = g->seg_tiles[t.seg];
+      r.off = t.off; r.count = t.count; r.seg = t.seg; r.need = g->seg_tiles[t.seg] + missing_tiles;
       // the segment's first tile: the previous entry belongs to another segment
       r.first = (!g->rtiles.empty() && g->rtiles.back().seg == t.seg) ? g->rtiles.back().first
                                                                       : (int)g->rtiles.size();
@@ -101,7 +107,7 @@ int validate_config(const qadam_config* c) {
   if (c->kg < -1 || c->kx < -1 || c->kx > 14) return QADAM_ERR_LEVEL;
   if (c->kg >= 0 && grad_levels(c->kg, c->grid_g) < 0) return QADAM_ERR_LEVEL;
   if (c->kg < 0 && c->grid_g != QADAM_GRID_POW2 && c->grid_g != QADAM_GRID_UNIFORM)
-    return QADAM_ERR_LEVEL;
+    return QADAM_ERR_LEVEL;      // the stochastic operator has no identity form
   if (!(c->beta1 >= 0.0f && c->beta1 < 1.0f) || !(c->beta2 >= 0.0f && c->beta2 < 1.0f) ||
       !(c->eps > 0.0f) || !std::isfinite(c->eps) || !std::isfinite(c->lr))
     return QADAM_ERR_HYPER;
@@ -150,7 +156,8 @@ int build_geometry(const qadam_config* c, Geometry* g) {
   } else {
     g->L = grad_levels(c->kg, c->grid_g);
     g->gbits = bits_for(2 * g->L + 1);
-    g->gmode = c->kg == 0 ? G_TERNARY : c->kg == 1 ? G_FIVE
+    g->gmode = c->grid_g == QADAM_GRID_STOCHASTIC ? G_STOCHASTIC
+             : c->kg == 0 ? G_TERNARY : c->kg == 1 ? G_FIVE
              : c->grid_g == QADAM_GRID_POW2 ? G_POW2 : G_UNIFORM;
   }
   g->xbits = c->kx < 0 ? 0 : c->kx + 2;
@@ -199,8 +206,11 @@ struct qadam_ctx {
   // persistent pipelined server pass (ternary codes): stages > 0 when in use
   float lambda = 0.0f;       // l2 term (qadam_set_regularization)
   int pipe_stages = 0;
-  int pipe_skip_16ths = 2;   // zero skipping while at most this many sixteenths of the workers are live
   size_t pipe_smem = 0;
+  int pipe_scale_cache = 0;  // bytes of the scales table the pipelined pass keeps in shared memory
+  qadam_options opt = {};
+  unsigned spin_limit = kSpinLimit;
+  bool range_open = false;   // a range of the current step has been served (qadam_server_step_range)
   CUtensorMap codes_map;
   unsigned* d_done = nullptr;
   // on-chip worker kernel (moments on the server, all workers in one call): grid > 0 when in use
@@ -247,6 +257,7 @@ WorkerKernel pick_quantize(const qadam_ctx* c) {
   if (!w && c->lambda != 0.0f) {
     // moments on the server: phase 2 forms u = g + e again, l2 term included
     switch (c->geo.gmode) {
+      case G_STOCHASTIC: return worker_quantize_kernel<false, G_STOCHASTIC, true>;
       case G_TERNARY: return worker_quantize_kernel<false, G_TERNARY, true>;
       case G_FIVE:    return worker_quantize_kernel<false, G_FIVE, true>;
       case G_POW2:    return worker_quantize_kernel<false, G_POW2, true>;
@@ -254,6 +265,7 @@ WorkerKernel pick_quantize(const qadam_ctx* c) {
     }
   }
   switch (c->geo.gmode) {
+    case G_STOCHASTIC: return w ? worker_quantize_kernel<true, G_STOCHASTIC> : worker_quantize_kernel<false, G_STOCHASTIC>;
     case G_TERNARY: return w ? worker_quantize_kernel<true, G_TERNARY> : worker_quantize_kernel<false, G_TERNARY>;
     case G_FIVE:    return w ? worker_quantize_kernel<true, G_FIVE>    : worker_quantize_kernel<false, G_FIVE>;
     case G_POW2:    return w ? worker_quantize_kernel<true, G_POW2>    : worker_quantize_kernel<false, G_POW2>;
@@ -264,6 +276,7 @@ WorkerKernel pick_quantize(const qadam_ctx* c) {
 ServerKernel pick_server(const qadam_ctx* c) {
   const bool s = c->cfg.placement == QADAM_PLACE_SERVER;
   switch (c->geo.gmode) {
+    case G_STOCHASTIC:
     case G_TERNARY:  return s ? server_step_kernel<true, G_TERNARY>  : server_step_kernel<false, G_TERNARY>;
     case G_FIVE:     return s ? server_step_kernel<true, G_FIVE>     : server_step_kernel<false, G_FIVE>;
     case G_POW2:     return s ? server_step_kernel<true, G_POW2>     : server_step_kernel<false, G_POW2>;
@@ -288,7 +301,8 @@ PipeKernel pick_pipe_n(int n) {
 PipeKernel pick_pipe(const qadam_ctx* c) {
   const bool sm = c->cfg.placement == QADAM_PLACE_SERVER;
   if (c->geo.gmode == G_FIVE) return sm ? pick_pipe_n<true, 3>(c->cfg.n) : pick_pipe_n<false, 3>(c->cfg.n);
-  if (c->geo.gmode == G_TERNARY) return sm ? pick_pipe_n<true, 2>(c->cfg.n) : pick_pipe_n<false, 2>(c->cfg.n);
+  if (c->geo.gmode == G_TERNARY || c->geo.gmode == G_STOCHASTIC)
+    return sm ? pick_pipe_n<true, 2>(c->cfg.n) : pick_pipe_n<false, 2>(c->cfg.n);
   // any other grid of at most 8 bits: table decode, worker count at run time
   return sm ? server_pipe_kernel<true, 0, 0> : server_pipe_kernel<false, 0, 0>;
 }
@@ -328,10 +342,13 @@ bool l2_split(const qadam_ctx* c) {
 }
 
 // grids of the split worker kernels (they depend on whether the l2 term is on)
-void plan_worker_grids(qadam_ctx* c) {
-  c->grid_absmax = resident_grid(pick_absmax(c), 0, c->sm_count);
-  c->grid_quant = resident_grid(pick_quantize(c), 0, c->sm_count);
-  c->grid_ident = resident_grid(pick_identity(c), 0, c->sm_count);
+bool plan_worker_grids(qadam_ctx* c) {
+  const int a = resident_grid(pick_absmax(c), 0, c->sm_count);
+  const int q = resident_grid(pick_quantize(c), 0, c->sm_count);
+  const int i = resident_grid(pick_identity(c), 0, c->sm_count);
+  if (a < 0 || q < 0 || i < 0) return false;
+  c->grid_absmax = a; c->grid_quant = q; c->grid_ident = i;
+  return true;
 }
 
 cudaEvent_t take_event(qadam_ctx* c) {
@@ -379,13 +396,14 @@ ServerParams make_server_params(const qadam_ctx* c, float alpha) {
   p.S = c->cfg.num_segments;
   p.n = c->cfg.n;
   p.k = c->cfg.kg; p.L = c->geo.L; p.gbits = c->geo.gbits;
-  p.gmode = c->geo.gmode;
+  p.gmode = c->geo.gmode == G_STOCHASTIC ? G_TERNARY : c->geo.gmode;   // stochastic codes are ternary codes
   p.kx = c->cfg.kx; p.xbits = c->geo.xbits;
   p.alpha = alpha;
   p.nf = (float)c->cfg.n;
   p.inv_nf = 1.0f / (float)c->cfg.n;
   p.status = c->buf.status;
   p.h = c->h;
+  p.spin_limit = c->spin_limit;
   return p;
 }
 
@@ -419,8 +437,20 @@ int qadam_query_sizes(const qadam_config* cfg, int64_t* D, int64_t* seg_off,
 }
 
 int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** out) {
+  return qadam_create_ex(cfg, b, nullptr, out);
+}
+
+int qadam_create_ex(const qadam_config* cfg, const qadam_buffers* b, const qadam_options* opt,
+                    qadam_ctx** out) {
   if (!cfg || !b || !out) return QADAM_ERR_NULL;
   *out = nullptr;
+  qadam_options o = {};
+  if (opt) o = *opt;
+  if ((o.server_kernel != QADAM_SERVER_AUTO && o.server_kernel != QADAM_SERVER_PLAIN) ||
+      (o.worker_kernel != QADAM_WORKER_AUTO && o.worker_kernel != QADAM_WORKER_STREAMING) ||
+      (o.hand_over != QADAM_HANDOVER_AUTO && o.hand_over != QADAM_HANDOVER_COUNTERS) ||
+      o.test_missing_tiles < 0 || o.reserved[0] || o.reserved[1] || o.reserved[2])
+    return QADAM_ERR_SIZE;
   qadam_ctx* c = new (std::nothrow) qadam_ctx();
   if (!c) return QADAM_ERR_CUDA;
   int rc = build_geometry(cfg, &c->geo);
@@ -437,6 +467,8 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
   if (!aligned(b->workspace, 256)) { delete c; return QADAM_ERR_ALIGN; }
   if (b->workspace_bytes < c->geo.workspace_bytes) { delete c; return QADAM_ERR_WORKSPACE; }
 
+  c->opt = o;
+  c->spin_limit = o.wait_polls ? o.wait_polls : kSpinLimit;
   c->cfg = *cfg;
   c->cfg.seg_len = nullptr;            // the caller's array is not kept; geo has a copy
   c->buf = *b;
@@ -463,7 +495,7 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
     delete c; return QADAM_ERR_CUDA;
   }
   c->server_smem = sizeof(float) * (size_t)cfg->n;
-  if (c->geo.gmode != G_TERNARY && c->geo.gmode != G_IDENTITY)
+  if (c->geo.gmode != G_TERNARY && c->geo.gmode != G_STOCHASTIC && c->geo.gmode != G_IDENTITY)
     c->server_smem += sizeof(float) * (size_t)cfg->n * ((size_t)1 << c->geo.gbits);
   if (c->server_smem > 200 * 1024) { delete c; return QADAM_ERR_SIZE; }
   ServerKernel sk = pick_server(c);
@@ -480,21 +512,22 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
     }
     const bool sm_mom = cfg->placement == QADAM_PLACE_SERVER;
     const bool table = c->geo.gmode == G_POW2 || c->geo.gmode == G_UNIFORM;
-    const bool pipe_codes = c->geo.gmode == G_TERNARY || c->geo.gmode == G_FIVE || (table && c->geo.gbits <= 8);
+    const bool pipe_codes = c->geo.gmode == G_TERNARY || c->geo.gmode == G_STOCHASTIC || c->geo.gmode == G_FIVE ||
+                            (table && c->geo.gbits <= 8);
     const size_t sb = pipe_stage_bytes(cfg->n, sm_mom, pipe_codes ? c->geo.gbits : 2);
-    const size_t head = pipe_head_bytes(table);
-    const char* env = std::getenv("QADAM_SERVER_KERNEL");
-    const bool want_plain = env && std::strcmp(env, "plain") == 0;
+    const size_t scale_cache = pipe_scale_cache_bytes(cfg->n, cfg->num_segments);
+    const size_t head = pipe_head_bytes(table, scale_cache);
+    const bool want_plain = o.server_kernel == QADAM_SERVER_PLAIN;
     int stages = (int)(((size_t)max_smem - head) / sb);
     stages = pipe_legal_stages(std::min(stages, kPipeMaxStages));
-    if (!want_plain && pipe_codes && cfg->n <= kPipeMaxWorkers && stages >= 2 &&
+    // the tensor copy addresses a tile's codes by a 32-bit coordinate in words of the stream
+    // (32-bit words, 64-bit for the table decode): longer streams take the plain kernel
+    const bool coord_fits = (long long)c->geo.gcode_bytes / (table ? 8 : 4) < (1ll << 31);
+    if (!want_plain && pipe_codes && coord_fits && cfg->n <= kPipeMaxWorkers && stages >= 2 &&
         make_codes_tensor_map(&c->codes_map, b->gcodes, (long long)c->geo.gcode_bytes, cfg->n,
                               c->geo.gbits, table)) {
       c->pipe_stages = stages;
-      if (const char* sk16 = std::getenv("QADAM_SKIP_16THS")) {
-        const int v = std::atoi(sk16);
-        if (v >= 0 && v <= 16) c->pipe_skip_16ths = v;
-      }
+      c->pipe_scale_cache = (int)scale_cache;
       c->pipe_smem = head + (size_t)stages * sb;
       if (!cuda_ok(cudaFuncSetAttribute(pick_pipe(c), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)c->pipe_smem))) {
@@ -502,7 +535,7 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
       }
     }
   }
-  plan_worker_grids(c);
+  if (!plan_worker_grids(c)) { delete c; return QADAM_ERR_CUDA; }
   c->grid_server = resident_grid(sk, c->server_smem, c->sm_count);
   c->grid_bcast = resident_grid(weight_broadcast_kernel, 0, c->sm_count);
   // Worker side, all workers in one call.  Segments small enough to be held by the
@@ -512,28 +545,24 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
   // plain streaming launches, over a tile table of their own.  The on-chip kernel needs
   // every CTA resident at once (its store side waits for other CTAs' load sides): one
   // CTA per SM, launched cooperatively.
-  // QADAM_WORKER_KERNEL=split: streaming launches only.
   {
     int coop = 0, max_smem = 0;
-    const char* env = std::getenv("QADAM_WORKER_KERNEL");
-    const bool want_split = env && std::strcmp(env, "split") == 0;
+    const bool want_split = o.worker_kernel == QADAM_WORKER_STREAMING;
     const bool wm = cfg->placement == QADAM_PLACE_WORKER;
-    const bool eligible = !want_split && c->geo.gmode != G_IDENTITY &&
+    // (the stochastic operator runs in the streaming launches only)
+    const bool eligible = !want_split && c->geo.gmode != G_IDENTITY && c->geo.gmode != G_STOCHASTIC &&
         cuda_ok(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev)) && coop &&
         cuda_ok(cudaDeviceGetAttribute(&max_smem, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
     if (eligible) {
       // the CTA's shared memory: a ring of slots for u and a few stages for e (227 KB: 14 in all)
-      const char* ee = std::getenv("QADAM_RESIDENT_ESTAGES");
-      int estages = ee ? std::atoi(ee) : 2;
-      estages = std::max(2, std::min(estages, kRMaxEStages));
+      const int estages = 2;                  // measured: 12 slots + 2 stages beat 11 + 3 and 10 + 4
       const int slots = std::min(((int)max_smem - kRHeadBytes - estages * resident_stage_bytes(wm)) / kRSlotBytes,
                                  kRMaxSlots);
       // a pair may give a CTA at most slots - 2 tiles: the rest of the ring lets the load side
       // run ahead into the next pair while this one is quantized and stored
-      const char* me = std::getenv("QADAM_RESIDENT_SPARE");
-      const int spare = std::max(1, me ? std::atoi(me) : 2);
+      const int spare = 2;
       if (slots - spare >= 1) {
-        build_resident((long long)c->sm_count * (slots - spare), &c->geo);
+        build_resident((long long)c->sm_count * (slots - spare), o.test_missing_tiles, &c->geo);
         c->res_slots = slots;
         c->res_estages = estages;
         c->res_smem = resident_smem_bytes(slots, estages, wm);
@@ -550,8 +579,7 @@ int qadam_create(const qadam_config* cfg, const qadam_buffers* b, qadam_ctx** ou
       }
     }
   }
-  if (c->grid_absmax < 0 || c->grid_quant < 0 || c->grid_ident < 0 || c->grid_server < 0 ||
-      c->grid_bcast < 0) {
+  if (c->grid_server < 0 || c->grid_bcast < 0) {
     delete c; return QADAM_ERR_CUDA;
   }
 
@@ -614,6 +642,33 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
   p.wcodes = static_cast<const unsigned char*>(c->buf.wcodes);
   p.kx = c->cfg.kx; p.xbits = c->geo.xbits;
   p.lambda = c->lambda;
+  p.spin_limit = c->spin_limit;
+  p.seed_lo = (unsigned)c->cfg.seed;
+  p.seed_hi = (unsigned)(c->cfg.seed >> 32);
+  p.step = (unsigned)step;
+
+  // the two streaming launches over a tile table: max-abs, then quantize
+  auto streaming = [&](const Tile* tiles, int tiles_per_worker) -> int {
+    WorkerParams q = p;
+    q.tiles = tiles;
+    q.tiles_per_worker = tiles_per_worker;
+    q.total_tiles = (long long)worker_count * tiles_per_worker;
+    int grid = (int)std::min<int64_t>(c->grid_absmax, q.total_tiles);
+    {
+      LaunchTimer lt(c, QADAM_K_ABSMAX);
+      pick_absmax(c)<<<grid, kThreads, 0, c->stream>>>(q);
+    }
+    if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
+    c->launches += 1;
+    grid = (int)std::min<int64_t>(c->grid_quant, q.total_tiles);
+    {
+      LaunchTimer lt(c, QADAM_K_QUANTIZE);
+      pick_quantize(c)<<<grid, kThreads, 0, c->stream>>>(q);
+    }
+    if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
+    c->launches += 1;
+    return QADAM_OK;
+  };
 
   if (c->geo.gmode == G_IDENTITY) {
     const int grid = (int)std::min<int64_t>(c->grid_ident, p.total_tiles);
@@ -623,71 +678,55 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
     }
     if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
     c->launches += 1;
-  } else if (c->grid_resident > 0 && worker_begin == 0 && worker_count == c->cfg.n && !l2_split(c)) {
-    const size_t pairs = (size_t)c->cfg.n * p.S;
-    if (!cuda_ok(cudaMemsetAsync(p.scale_bits, 0, sizeof(unsigned) * pairs, c->stream)) ||
-        !cuda_ok(cudaMemsetAsync(c->d_done, 0, sizeof(unsigned) * pairs, c->stream)))
-      return QADAM_ERR_CUDA;
-    const bool l2 = c->lambda != 0.0f;
-    const bool use_words = !l2 && c->d_words != nullptr && c->grid_resident <= kWordCtas &&
-                           std::getenv("QADAM_RESIDENT_COUNTERS") == nullptr;
-    if (use_words &&
-        !cuda_ok(cudaMemsetAsync(c->d_words, 0, sizeof(unsigned long long) * pairs * c->grid_resident, c->stream)))
-      return QADAM_ERR_CUDA;
-    WorkerResidentParams rp;
-    rp.w = p;
-    rp.words = use_words ? c->d_words : nullptr;
-    rp.rtiles = c->d_rtiles;
-    rp.done = c->d_done;
-    rp.TR = (int)c->geo.rtiles.size();
-    rp.total = (long long)c->cfg.n * rp.TR;
-    rp.slots = c->res_slots;
-    rp.estages = c->res_estages;
-    void* args[] = {&rp};
-    cudaError_t e;
-    {
-      LaunchTimer lt(c, QADAM_K_WORKER_FUSED);
-      e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(pick_worker_resident(c, l2, use_words)),
-                                      dim3(c->grid_resident), dim3(kRThreads), args, c->res_smem, c->stream);
-    }
-    if (!cuda_ok(e)) return QADAM_ERR_CUDA;
-    c->launches += 1;
-    if (!c->geo.btiles.empty()) {
-      // the segments too large for the chip: two streaming passes over their own tile table
-      p.tiles = c->d_btiles;
-      p.tiles_per_worker = (int)c->geo.btiles.size();
-      p.total_tiles = (long long)worker_count * p.tiles_per_worker;
-      int grid = (int)std::min<int64_t>(c->grid_absmax, p.total_tiles);
-      {
-        LaunchTimer lt(c, QADAM_K_ABSMAX);
-        pick_absmax(c)<<<grid, kThreads, 0, c->stream>>>(p);
-      }
-      if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
-      grid = (int)std::min<int64_t>(c->grid_quant, p.total_tiles);
-      {
-        LaunchTimer lt(c, QADAM_K_QUANTIZE);
-        pick_quantize(c)<<<grid, kThreads, 0, c->stream>>>(p);
-      }
-      if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
-      c->launches += 2;
-    }
   } else {
+    // the scales of these workers start at zero (the kernels fold maxima into them)
     if (!cuda_ok(cudaMemsetAsync(p.scale_bits + (size_t)worker_begin * p.S, 0,
                                  sizeof(unsigned) * (size_t)worker_count * p.S, c->stream)))
       return QADAM_ERR_CUDA;
-    int grid = (int)std::min<int64_t>(c->grid_absmax, p.total_tiles);
-    {
-      LaunchTimer lt(c, QADAM_K_ABSMAX);
-      pick_absmax(c)<<<grid, kThreads, 0, c->stream>>>(p);
+    bool on_chip = c->grid_resident > 0 && worker_begin == 0 && worker_count == c->cfg.n && !l2_split(c);
+    if (on_chip) {
+      const size_t pairs = (size_t)c->cfg.n * p.S;
+      const bool l2 = c->lambda != 0.0f;
+      const bool use_words = !l2 && c->d_words != nullptr && c->grid_resident <= kWordCtas &&
+                             c->opt.hand_over == QADAM_HANDOVER_AUTO;
+      if (!cuda_ok(cudaMemsetAsync(c->d_done, 0, sizeof(unsigned) * pairs, c->stream)) ||
+          (use_words && !cuda_ok(cudaMemsetAsync(c->d_words, 0, sizeof(unsigned long long) * pairs * c->grid_resident,
+                                                 c->stream))))
+        return QADAM_ERR_CUDA;
+      WorkerResidentParams rp;
+      rp.w = p;
+      rp.words = use_words ? c->d_words : nullptr;
+      rp.rtiles = c->d_rtiles;
+      rp.done = c->d_done;
+      rp.TR = (int)c->geo.rtiles.size();
+      rp.total = (long long)c->cfg.n * rp.TR;
+      rp.slots = c->res_slots;
+      rp.estages = c->res_estages;
+      void* args[] = {&rp};
+      cudaError_t e;
+      {
+        LaunchTimer lt(c, QADAM_K_WORKER_FUSED);
+        e = cudaLaunchCooperativeKernel(reinterpret_cast<const void*>(pick_worker_resident(c, l2, use_words)),
+                                        dim3(c->grid_resident), dim3(kRThreads), args, c->res_smem, c->stream);
+      }
+      if (cuda_ok(e)) {
+        c->launches += 1;
+        if (!c->geo.btiles.empty()) {
+          // the segments too large for the chip: two streaming passes over their own tile table
+          const int rc = streaming(c->d_btiles, (int)c->geo.btiles.size());
+          if (rc != QADAM_OK) return rc;
+        }
+      } else {
+        // the cooperative launch was refused (the error is kept for qadam_last_cuda_error):
+        // nothing of it runs, and the streaming launches over the whole vector still can
+        (void)cudaGetLastError();
+        on_chip = false;
+      }
     }
-    if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
-    grid = (int)std::min<int64_t>(c->grid_quant, p.total_tiles);
-    {
-      LaunchTimer lt(c, QADAM_K_QUANTIZE);
-      pick_quantize(c)<<<grid, kThreads, 0, c->stream>>>(p);
+    if (!on_chip) {
+      const int rc = streaming(c->d_tiles, (int)c->geo.tiles.size());
+      if (rc != QADAM_OK) return rc;
     }
-    if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
-    c->launches += 2;
   }
   c->workers_done += worker_count;
   return QADAM_OK;
@@ -707,35 +746,110 @@ int qadam_set_regularization(qadam_ctx* c, float lambda) {
   if (!c) return QADAM_ERR_NULL;
   if (!(lambda >= 0.0f) || !std::isfinite(lambda)) return QADAM_ERR_HYPER;
   const bool changed = (c->lambda != 0.0f) != (lambda != 0.0f);
+  const float before = c->lambda;
   c->lambda = lambda;
-  if (changed) plan_worker_grids(c);
+  // the streaming kernels with and without the term differ: their grids are planned again
+  if (changed && !plan_worker_grids(c)) {
+    c->lambda = before;
+    return QADAM_ERR_CUDA;
+  }
   return QADAM_OK;
 }
 
-int qadam_server_step(qadam_ctx* c, int64_t step, float lr_t) {
-  if (!c) return QADAM_ERR_NULL;
-  if (step != c->last_server_step + 1 || c->workers_done < c->cfg.n) return QADAM_ERR_STEP;
-  const float alpha = lr_t < 0.0f ? c->cfg.lr : lr_t;
-  if (!std::isfinite(alpha)) return QADAM_ERR_HYPER;
-  const ServerParams p = make_server_params(c, alpha);
-  const int grid = (int)std::min<int64_t>(c->grid_server, (int64_t)c->geo.tiles.size());
+namespace {
+
+// Index of the tile that starts at element `elem` in a tile table sorted by offset
+// (tiles.size() for elem = D), or -1 when no tile starts there.
+long long tile_index_at(const std::vector<Tile>& tiles, int64_t D, int64_t elem) {
+  if (elem == D) return (long long)tiles.size();
+  auto it = std::lower_bound(tiles.begin(), tiles.end(), elem,
+                             [](const Tile& t, int64_t e) { return t.off < e; });
+  if (it == tiles.end() || it->off != elem) return -1;
+  return (long long)(it - tiles.begin());
+}
+
+// The server pass over tiles [tb, te) of the 4096-element table, which are ptiles
+// [pb, pe) of the 2048-element table.
+int launch_server(qadam_ctx* c, float alpha, long long tb, long long te, long long pb, long long pe) {
+  if (te <= tb) return QADAM_OK;
+  ServerParams p = make_server_params(c, alpha);
   {
     LaunchTimer lt(c, QADAM_K_SERVER);
     if (c->pipe_stages > 0) {
       const int n = c->cfg.n;
       const int inv_exact = (n & (n - 1)) == 0 ? 1 : 0;
-      const int np = (int)c->geo.ptiles.size();
+      const int np = (int)(pe - pb);
       const int pgrid = std::min(c->sm_count, np);
-      pick_pipe(c)<<<pgrid, kPipeThreads, c->pipe_smem, c->stream>>>(p, c->codes_map, c->d_ptiles, np,
-                                                                      c->pipe_stages, inv_exact, c->pipe_skip_16ths);
+      pick_pipe(c)<<<pgrid, kPipeThreads, c->pipe_smem, c->stream>>>(p, c->codes_map, c->d_ptiles + pb, np,
+                                                                      c->pipe_stages, inv_exact, c->pipe_scale_cache);
     } else {
+      p.tiles = c->d_tiles + tb;
+      p.tiles_per_worker = (int)(te - tb);
+      const int grid = (int)std::min<int64_t>(c->grid_server, te - tb);
       pick_server(c)<<<grid, kThreads, c->server_smem, c->stream>>>(p);
     }
   }
   if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
   c->launches += 1;
+  return QADAM_OK;
+}
+
+}  // namespace
+
+int qadam_server_step(qadam_ctx* c, int64_t step, float lr_t) {
+  if (!c) return QADAM_ERR_NULL;
+  if (step != c->last_server_step + 1 || c->workers_done < c->cfg.n || c->range_open) return QADAM_ERR_STEP;
+  const float alpha = lr_t < 0.0f ? c->cfg.lr : lr_t;
+  if (!std::isfinite(alpha)) return QADAM_ERR_HYPER;
+  const int rc = launch_server(c, alpha, 0, (long long)c->geo.tiles.size(), 0, (long long)c->geo.ptiles.size());
+  if (rc != QADAM_OK) return rc;
   c->last_server_step = step;
   c->workers_done = 0;
+  return QADAM_OK;
+}
+
+int qadam_server_step_range(qadam_ctx* c, int64_t step, float lr_t, int64_t elem_begin, int64_t elem_end) {
+  if (!c) return QADAM_ERR_NULL;
+  if (step != c->last_server_step + 1) return QADAM_ERR_STEP;
+  const float alpha = lr_t < 0.0f ? c->cfg.lr : lr_t;
+  if (!std::isfinite(alpha)) return QADAM_ERR_HYPER;
+  if (elem_begin < 0 || elem_end < elem_begin || elem_end > c->geo.D) return QADAM_ERR_SIZE;
+  const long long tb = tile_index_at(c->geo.tiles, c->geo.D, elem_begin);
+  const long long te = tile_index_at(c->geo.tiles, c->geo.D, elem_end);
+  const long long pb = tile_index_at(c->geo.ptiles, c->geo.D, elem_begin);
+  const long long pe = tile_index_at(c->geo.ptiles, c->geo.D, elem_end);
+  if (tb < 0 || te < 0 || pb < 0 || pe < 0) return QADAM_ERR_SIZE;
+  const int rc = launch_server(c, alpha, tb, te, pb, pe);
+  if (rc != QADAM_OK) return rc;
+  c->range_open = true;
+  return QADAM_OK;
+}
+
+int qadam_finish_step(qadam_ctx* c, int64_t step) {
+  if (!c) return QADAM_ERR_NULL;
+  if (step != c->last_server_step + 1) return QADAM_ERR_STEP;
+  c->last_server_step = step;
+  c->workers_done = 0;
+  c->range_open = false;
+  return QADAM_OK;
+}
+
+int qadam_shard_cuts(const qadam_config* cfg, int32_t shards, int64_t* cuts) {
+  if (!cfg || !cuts) return QADAM_ERR_NULL;
+  if (shards < 1) return QADAM_ERR_SIZE;
+  Geometry geo;
+  const int rc = build_geometry(cfg, &geo);
+  if (rc != QADAM_OK) return rc;
+  // cut g: the first tile whose start is at or beyond g * D / shards
+  const std::vector<Tile>& tiles = geo.tiles;
+  cuts[0] = 0;
+  for (int32_t g = 1; g < shards; ++g) {
+    const int64_t want = (int64_t)(((__int128)geo.D * g) / shards);
+    auto it = std::lower_bound(tiles.begin(), tiles.end(), want,
+                               [](const Tile& t, int64_t e) { return t.off < e; });
+    cuts[g] = it == tiles.end() ? geo.D : it->off;
+  }
+  cuts[shards] = geo.D;
   return QADAM_OK;
 }
 
@@ -743,7 +857,9 @@ int qadam_step_host(qadam_ctx* c, int64_t step, const float* g_host, float* g_st
                     void* out_host, float lr_t) {
   if (!c || !g_host || !g_stage) return QADAM_ERR_NULL;
   if (!aligned(g_stage, 16)) return QADAM_ERR_ALIGN;
-  if (step != c->last_server_step + 1 || c->workers_done != 0) return QADAM_ERR_STEP;
+  if (step != c->last_server_step + 1 || c->workers_done != 0 || c->range_open) return QADAM_ERR_STEP;
+  const float alpha = lr_t < 0.0f ? c->cfg.lr : lr_t;
+  if (!std::isfinite(alpha)) return QADAM_ERR_HYPER;
   const size_t gbytes = sizeof(float) * (size_t)c->cfg.n * (size_t)c->geo.D;
   if (!cuda_ok(cudaMemcpyAsync(g_stage, g_host, gbytes, cudaMemcpyHostToDevice, c->stream)))
     return QADAM_ERR_CUDA;

@@ -31,7 +31,9 @@ enum GMode : int {
   G_FIVE = 1,      // {0, 1/2, 1}                (kg = 1, either grid)
   G_POW2 = 2,      // {0, 2^-k, ..., 1}          (kg >= 2, geometric)
   G_UNIFORM = 3,   // {0, 1/2^k, 2/2^k, ..., 1}  (kg >= 2, uniform)
-  G_IDENTITY = 4   // Q_g = identity
+  G_IDENTITY = 4,  // Q_g = identity
+  G_STOCHASTIC = 5 // {0, 1} chosen at random with probability |u| / |u|_inf (worker side only:
+                   // the codes it emits are ternary codes and are decoded as such)
 };
 
 struct Hyper {
@@ -108,34 +110,98 @@ __device__ __forceinline__ float level_value(int c, int k) {
   }
 }
 
+// What Q_g needs of a segment's scale s = |u|_inf, computed once per tile rather than per
+// coordinate.  The level of a coordinate is decided by y = fl(|u| / s) against the midpoints
+// of G; the fast paths below settle that decision without dividing for all but a sliver of
+// values and fall back to the division inside the sliver, so the result is always the one
+// the division gives.
+struct GradScale {
+  float s;
+  float inv;      // fl(1 / s), times 2^k for the uniform grid
+  float half;     // ternary: s / 2 (exact) and the upper end of the sliver above it
+  float half_hi;
+  bool fast;      // s is an ordinary number (not zero, tiny, Inf or NaN): the fast paths apply
+};
+template <int MODE>
+__device__ __forceinline__ GradScale grad_scale(float s, int k) {
+  GradScale g;
+  g.s = s;
+  g.fast = s >= 1e-30f && s < 3.0e38f;
+  g.half = __fmul_rn(0.5f, s);
+  g.half_hi = __fmul_rn(g.half, 1.000000476837158203125f);          // 1 + 2^-21
+  g.inv = 0.0f;
+  if constexpr (MODE == G_FIVE || MODE == G_POW2 || MODE == G_UNIFORM) {
+    if (g.fast) {
+      g.inv = __fdiv_rn(1.0f, s);
+      if constexpr (MODE == G_UNIFORM) g.inv = __fmul_rn(g.inv, exp2i(k));      // exact
+    }
+  }
+  return g;
+}
+
 // One coordinate of Q_g and of the error update:  given u and the segment's scale
 // s = |u|_inf, returns the code (level index + L) and writes e' = u - Q_g(u).
 template <int MODE>
-__device__ __forceinline__ unsigned quantize_grad(float u, float s, int k, int L, float& e_next) {
+__device__ __forceinline__ unsigned quantize_grad(float u, const GradScale& gs, int k, int L, float& e_next) {
+  const float s = gs.s;
+  const float a = fabsf(u);
+  const bool neg = u < 0.0f;
   if constexpr (MODE == G_TERNARY) {
-    // The decision is y = fl(|u| / s) > 1/2.  It is settled without dividing for all but
-    // a sliver of values: |u| <= s/2 gives a quotient <= 1/2 (s/2 is exact for a normal
-    // s), and |u| > (s/2)(1 + 2^-21) gives a quotient whose rounding stays above 1/2.
-    // Only values inside that band, and tiny or non-finite scales, take the division.
-    const float a = fabsf(u);
-    const float h = __fmul_rn(0.5f, s);
-    const float hi = __fmul_rn(h, 1.000000476837158203125f);       // 1 + 2^-21
+    // The decision is y = fl(|u| / s) > 1/2.  |u| <= s/2 gives a quotient <= 1/2 (s/2 is exact
+    // for a normal s), and |u| > (s/2)(1 + 2^-21) gives a quotient whose rounding stays above
+    // 1/2.  Only values inside that band, and tiny or non-finite scales, take the division.
     bool one;
-    if (a <= h && s >= 1e-30f) {
+    if (a <= gs.half && gs.fast) {
       one = false;
-    } else if (a > hi && s >= 1e-30f && s < 3.0e38f) {
+    } else if (a > gs.half_hi && gs.fast) {
       one = true;
     } else {
       one = __fdiv_rn(a, s) > 0.5f;
     }
-    const bool neg = u < 0.0f;
     const float deq = one ? (neg ? -s : s) : 0.0f;
     e_next = __fsub_rn(u, deq);
     return one ? (neg ? 0u : 2u) : 1u;
   }
-  const float y = __fdiv_rn(fabsf(u), s);
-  const int c = level_index<MODE>(y, k, L);
-  const bool neg = u < 0.0f;
+  int c;
+  bool decided = false;
+  if constexpr (MODE == G_FIVE || MODE == G_POW2) {
+    // Geometric levels 0, 2^-k, ..., 1: the midpoints are 2^(-k-1) and 1.5 * 2^j, so the level
+    // index is read off the exponent of y and of whether its fraction reaches 1.5.
+    // y' = fl(|u| * fl(1/s)) is within 2^-22 (relative) of y; unless y' lies within 2^-19 of a
+    // midpoint (fraction near 1 or near 1.5) both give the same index.
+    const int kk = MODE == G_FIVE ? 1 : k;
+    if (gs.fast) {
+      const float yp = __fmul_rn(a, gs.inv);
+      const unsigned yb = __float_as_uint(yp);
+      const unsigned m = yb & 0x7fffffu;
+      const bool near = (m - 0x3ffff0u) <= 0x20u || m <= 0x10u || m >= 0x7fffefu;
+      if (!near) {
+        const int e15 = (int)((yb + 0x00400000u) >> 23) - 127;      // exponent, plus one when the fraction is >= 1.5
+        const int upper = e15 + kk;
+        c = (yp > exp2i(-kk - 1) ? 1 : 0) + (upper > 0 ? upper : 0);
+        c = c > L ? L : c;
+        decided = true;
+      }
+    }
+  } else if constexpr (MODE == G_UNIFORM) {
+    // Uniform levels c / 2^k: the index is ceil(z - 1/2) with z = y 2^k.  z' = |u| * fl(2^k / s)
+    // is within 2^-22 (relative) of z; unless z' - 1/2 lies within 2^-15 of an integer (z <= 64)
+    // both give the same index.
+    if (gs.fast) {
+      const float t = __fadd_rn(__fmul_rn(a, gs.inv), -0.5f);
+      const float ct = ceilf(t);
+      const float w = __fsub_rn(ct, t);                              // in [0, 1)
+      if (w > 6.1035156e-05f && w < 0.99993896f) {
+        c = (int)ct;
+        c = c < 0 ? 0 : (c > L ? L : c);
+        decided = true;
+      }
+    }
+  }
+  if (!decided) {
+    const float y = __fdiv_rn(a, s);
+    c = level_index<MODE>(y, k, L);
+  }
   float deq = 0.0f;                                   // level 0 carries no sign
   if (c != 0) {
     const float mag = __fmul_rn(s, level_value<MODE>(c, k));
@@ -143,6 +209,38 @@ __device__ __forceinline__ unsigned quantize_grad(float u, float s, int k, int L
   }
   e_next = __fsub_rn(u, deq);
   return (unsigned)(neg ? L - c : L + c);
+}
+
+// Philox4x32-10 (Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3",
+// SC 2011), from its published definition: ten rounds over a counter of four 32-bit words
+// under a key of two; a round multiplies words 0 and 2 by fixed odd constants, keeps both
+// halves of the products and mixes in the other words and the key; the key words grow by two
+// Weyl constants after every round.
+__device__ __forceinline__ uint4 philox4x32_10(uint4 c, uint2 k) {
+#pragma unroll
+  for (int round = 0; round < 10; ++round) {
+    const unsigned hi0 = __umulhi(0xD2511F53u, c.x), lo0 = 0xD2511F53u * c.x;
+    const unsigned hi1 = __umulhi(0xCD9E8D57u, c.z), lo1 = 0xCD9E8D57u * c.z;
+    c = make_uint4(hi1 ^ c.y ^ k.x, lo1, hi0 ^ c.w ^ k.y, lo0);
+    k.x += 0x9E3779B9u;
+    k.y += 0xBB67AE85u;
+  }
+  return c;
+}
+
+// One coordinate of the stochastic ternary operator (the method Section 5.1 compares with):
+// level 1 with probability y = fl(|u| / s), decided by r < y with r the top 24 bits of the
+// coordinate's random word times 2^-24; returns the code and writes e' = u - Q(u).
+__device__ __forceinline__ unsigned quantize_grad_stochastic(float u, float s, unsigned word, float& e_next) {
+  bool one = false;
+  if (s > 0.0f) {
+    const float r = __fmul_rn((float)(word >> 8), 5.9604644775390625e-08f);    // exact
+    one = r < __fdiv_rn(fabsf(u), s);
+  }
+  const bool neg = u < 0.0f;
+  const float deq = one ? (neg ? -s : s) : 0.0f;
+  e_next = __fsub_rn(u, deq);
+  return one ? (neg ? 0u : 2u) : 1u;
 }
 
 // One coordinate of Q_x (Section 5.1): nearest point of the grid c / 2^(kx+1),

@@ -36,6 +36,9 @@ struct WorkerParams {
   const unsigned char* wcodes;  // packed Q_x(x) (kx >= 0)
   int kx, xbits;
   float lambda;
+  unsigned spin_limit;          // persistent kernels: polls of one wait before it gives up
+  // stochastic operator: key of the random stream and the step number
+  unsigned seed_lo, seed_hi, step;
 };
 
 // Packed weight codes of at most 8 bits: the two 32-bit words that hold this lane's 4 codes
@@ -141,6 +144,7 @@ struct ServerParams {
   float inv_nf;          // 1/n, exact when n is a power of two
   unsigned* status;
   Hyper h;
+  unsigned spin_limit;   // pipelined pass: polls of one wait before it gives up
 };
 
 __device__ __forceinline__ float4 ld_f4(const float* p) {
@@ -253,55 +257,83 @@ template <bool U_IN_E, int MODE, bool L2 = false>
 __global__ void __launch_bounds__(kThreads)
 worker_quantize_kernel(const WorkerParams p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  for (long long t = blockIdx.x; t < p.total_tiles; t += gridDim.x) {
-    const int wl = (int)(t / p.tiles_per_worker);
-    const Tile tile = p.tiles[(int)(t - (long long)wl * p.tiles_per_worker)];
-    const int w = p.worker_begin + wl;
-    const unsigned sb = p.scale_bits[(long long)w * p.S + tile.seg];
-    const float s = __uint_as_float(sb);
-    if (sb >= 0x7f800000u && threadIdx.x == 0) atomicOr(p.status, 1u);
-    const float* gp = p.g + (long long)wl * p.D + tile.off;
-    const long long so = (long long)w * p.D + tile.off;
-    unsigned char* cw = p.gcodes + (long long)w * p.gcode_bytes;
-    float4 gv[kRows], ev[kRows];
-    bool act[kRows];
+  // With u left in e's slot a tile brings only one array in, so two tiles are taken per
+  // round to keep as many loads in flight as the two-array form has.
+  constexpr int kPerRound = U_IN_E ? 2 : 1;
+  for (long long t0 = blockIdx.x; t0 < p.total_tiles; t0 += (long long)kPerRound * gridDim.x) {
+    Tile tile[kPerRound];
+    int wl[kPerRound];
+    bool have[kPerRound];
+    float4 gv[kPerRound][kRows], ev[kPerRound][kRows];
 #pragma unroll
-    for (int r = 0; r < kRows; ++r) {
-      const int idx = r * kRowElems + threadIdx.x * 4;
-      act[r] = idx < tile.count;
-      if (act[r]) {
-        if constexpr (!U_IN_E) gv[r] = ld_f4_stream(gp + idx);
-        ev[r] = ld_f4(p.e + so + idx);
+    for (int a = 0; a < kPerRound; ++a) {
+      const long long t = t0 + (long long)a * gridDim.x;
+      have[a] = t < p.total_tiles;
+      if (!have[a]) continue;
+      wl[a] = (int)(t / p.tiles_per_worker);
+      tile[a] = p.tiles[(int)(t - (long long)wl[a] * p.tiles_per_worker)];
+      const float* gp = p.g + (long long)wl[a] * p.D + tile[a].off;
+      const long long so = (long long)(p.worker_begin + wl[a]) * p.D + tile[a].off;
+#pragma unroll
+      for (int r = 0; r < kRows; ++r) {
+        const int idx = r * kRowElems + threadIdx.x * 4;
+        if (idx < tile[a].count) {
+          if constexpr (!U_IN_E) gv[a][r] = ld_f4_stream(gp + idx);
+          ev[a][r] = ld_f4(p.e + so + idx);
+        }
       }
     }
 #pragma unroll
-    for (int r = 0; r < kRows; ++r) {
-      if (!act[r]) continue;                    // warp-uniform: counts are multiples of 128
-      const int idx = r * kRowElems + threadIdx.x * 4;
-      float ee[4] = {ev[r].x, ev[r].y, ev[r].z, ev[r].w};
-      float uu[4];
-      if constexpr (U_IN_E) {
+    for (int a = 0; a < kPerRound; ++a) {
+      if (!have[a]) continue;
+      const int w = p.worker_begin + wl[a];
+      const unsigned sb = p.scale_bits[(long long)w * p.S + tile[a].seg];
+      const float s = __uint_as_float(sb);
+      const GradScale gs = grad_scale<MODE == G_STOCHASTIC ? G_TERNARY : MODE>(s, p.k);
+      if (sb >= 0x7f800000u && threadIdx.x == 0) atomicOr(p.status, 1u);
+      const long long so = (long long)w * p.D + tile[a].off;
+      unsigned char* cw = p.gcodes + (long long)w * p.gcode_bytes;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) uu[c] = ee[c];
-      } else {
-        float gg[4] = {gv[r].x, gv[r].y, gv[r].z, gv[r].w};
-        if constexpr (L2) add_l2_term(p, tile.off + r * kRowElems + warp * 128, lane, gg);
+      for (int r = 0; r < kRows; ++r) {
+        const int idx = r * kRowElems + threadIdx.x * 4;
+        if (idx >= tile[a].count) continue;         // warp-uniform: counts are multiples of 128
+        float ee[4] = {ev[a][r].x, ev[a][r].y, ev[a][r].z, ev[a][r].w};
+        float uu[4];
+        if constexpr (U_IN_E) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) uu[c] = __fadd_rn(gg[c], ee[c]);
-      }
-      unsigned code[4];
-      float en[4];
+          for (int c = 0; c < 4; ++c) uu[c] = ee[c];
+        } else {
+          float gg[4] = {gv[a][r].x, gv[a][r].y, gv[a][r].z, gv[a][r].w};
+          if constexpr (L2) add_l2_term(p, tile[a].off + r * kRowElems + warp * 128, lane, gg);
 #pragma unroll
-      for (int c = 0; c < 4; ++c) code[c] = quantize_grad<MODE>(uu[c], s, p.k, p.L, en[c]);
-      st_f4(p.e + so + idx, make_float4(en[0], en[1], en[2], en[3]));
-      const long long row_elem = tile.off + r * kRowElems + warp * 128;
-      void* dst = cw + row_elem * p.bits / 8;
-      if constexpr (MODE == G_TERNARY) {
-        pack_row_store<2>(code[0], code[1], code[2], code[3], dst, lane);
-      } else if constexpr (MODE == G_FIVE) {
-        pack_row_store<3>(code[0], code[1], code[2], code[3], dst, lane);
-      } else {
-        pack_row_store_rt(p.bits, code[0], code[1], code[2], code[3], dst, lane);
+          for (int c = 0; c < 4; ++c) uu[c] = __fadd_rn(gg[c], ee[c]);
+        }
+        unsigned code[4];
+        float en[4];
+        if constexpr (MODE == G_STOCHASTIC) {
+          // the four coordinates of this thread are one block of the stream: counter
+          // (element / 4, worker, step), key = seed
+          const unsigned long long block = (unsigned long long)(tile[a].off + idx) >> 2;
+          const uint4 rnd = philox4x32_10(make_uint4((unsigned)block, (unsigned)(block >> 32), (unsigned)w, p.step),
+                                          make_uint2(p.seed_lo, p.seed_hi));
+          code[0] = quantize_grad_stochastic(uu[0], s, rnd.x, en[0]);
+          code[1] = quantize_grad_stochastic(uu[1], s, rnd.y, en[1]);
+          code[2] = quantize_grad_stochastic(uu[2], s, rnd.z, en[2]);
+          code[3] = quantize_grad_stochastic(uu[3], s, rnd.w, en[3]);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 4; ++c) code[c] = quantize_grad<MODE>(uu[c], gs, p.k, p.L, en[c]);
+        }
+        st_f4(p.e + so + idx, make_float4(en[0], en[1], en[2], en[3]));
+        const long long row_elem = tile[a].off + r * kRowElems + warp * 128;
+        void* dst = cw + row_elem * p.bits / 8;
+        if constexpr (MODE == G_TERNARY || MODE == G_STOCHASTIC) {
+          pack_row_store<2>(code[0], code[1], code[2], code[3], dst, lane);
+        } else if constexpr (MODE == G_FIVE) {
+          pack_row_store<3>(code[0], code[1], code[2], code[3], dst, lane);
+        } else {
+          pack_row_store_rt(p.bits, code[0], code[1], code[2], code[3], dst, lane);
+        }
       }
     }
   }

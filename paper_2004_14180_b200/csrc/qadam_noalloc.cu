@@ -16,6 +16,7 @@
 
 #include <mutex>
 
+#include "qadam_host.h"
 #include "qadam_kernels.cuh"
 
 using namespace qadam;
@@ -34,21 +35,40 @@ constexpr size_t kScratchBytes = kAccBytes + sizeof(Tile) * (size_t)kStaticMaxTi
 static __device__ __align__(256) unsigned char g_static_scratch[kScratchBytes];
 
 constexpr int kMaxDevices = 64;
-void* g_scratch_addr[kMaxDevices] = {nullptr};     // device address of the array, per device
+struct DeviceSetup {
+  void* scratch = nullptr;   // device address of the array on this device
+  int grid = 0;              // CTAs that keep the device full with the max-abs kernel
+};
+DeviceSetup g_setup[kMaxDevices];
 std::mutex g_setup_mutex;
 
-// Device address of the scratch on the current device; looked up once per device.
-int scratch_for_current_device(void** out) {
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return QADAM_ERR_CUDA;
-  std::lock_guard<std::mutex> lock(g_setup_mutex);
-  if (g_scratch_addr[dev] == nullptr) {
-    void* ptr = nullptr;
-    const cudaError_t e = cudaGetSymbolAddress((void**)&ptr, g_static_scratch);
-    if (e != cudaSuccess || ptr == nullptr) return QADAM_ERR_CUDA;
-    g_scratch_addr[dev] = ptr;
+inline bool cuda_ok(cudaError_t e) {
+  if (e != cudaSuccess) {
+    record_cuda_error((int)e);
+    return false;
   }
-  *out = g_scratch_addr[dev];
+  return true;
+}
+
+// Address of the scratch and launch width on the current device; looked up once per
+// device, before anything is enqueued.
+int setup_for_current_device(DeviceSetup* out) {
+  int dev = 0;
+  if (!cuda_ok(cudaGetDevice(&dev))) return QADAM_ERR_CUDA;
+  if (dev < 0 || dev >= kMaxDevices) return QADAM_ERR_CAPACITY;
+  std::lock_guard<std::mutex> lock(g_setup_mutex);
+  DeviceSetup& d = g_setup[dev];
+  if (d.scratch == nullptr) {
+    void* ptr = nullptr;
+    int sms = 0, per_sm = 0;
+    if (!cuda_ok(cudaGetSymbolAddress((void**)&ptr, g_static_scratch)) || ptr == nullptr ||
+        !cuda_ok(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev)) ||
+        !cuda_ok(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, worker_absmax_kernel<false>, kThreads, 0)))
+      return QADAM_ERR_CUDA;
+    d.grid = sms * (per_sm > 0 ? per_sm : 1);
+    d.scratch = ptr;
+  }
+  *out = d;
   return QADAM_OK;
 }
 
@@ -80,9 +100,10 @@ extern "C" int qadam_worker_scales_static(const float* g, const float* e, int64_
   if ((reinterpret_cast<uintptr_t>(g) | reinterpret_cast<uintptr_t>(e)) % 16 != 0 ||
       reinterpret_cast<uintptr_t>(scales) % 4 != 0)
     return QADAM_ERR_ALIGN;
-  void* scratch = nullptr;
-  const int rc = scratch_for_current_device(&scratch);
+  DeviceSetup setup;
+  const int rc = setup_for_current_device(&setup);
   if (rc != QADAM_OK) return rc;
+  void* scratch = setup.scratch;
   cudaStream_t st = static_cast<cudaStream_t>(stream);
   unsigned* acc = static_cast<unsigned*>(scratch);
   Tile* tiles = reinterpret_cast<Tile*>(static_cast<unsigned char*>(scratch) + kAccBytes);
@@ -90,9 +111,9 @@ extern "C" int qadam_worker_scales_static(const float* g, const float* e, int64_
 
   // The array still holds the previous call's table and maxima: rewrite the table for
   // this D and clear the accumulators, which must start at zero.
-  if (cudaMemsetAsync(acc, 0, sizeof(unsigned) * (size_t)n, st) != cudaSuccess) return QADAM_ERR_CUDA;
+  if (!cuda_ok(cudaMemsetAsync(acc, 0, sizeof(unsigned) * (size_t)n, st))) return QADAM_ERR_CUDA;
   static_fill_tiles_kernel<<<(num_tiles + 255) / 256, 256, 0, st>>>(tiles, (long long)D, num_tiles);
-  if (cudaGetLastError() != cudaSuccess) return QADAM_ERR_CUDA;
+  if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
 
   WorkerParams p;
   p.g = g;
@@ -112,18 +133,14 @@ extern "C" int qadam_worker_scales_static(const float* g, const float* e, int64_
   p.alpha = 0.0f;
   p.h = Hyper{0.0f, 0.0f, 1.0f, 1.0f, 1.0f};
   p.x = nullptr; p.wcodes = nullptr; p.kx = -1; p.xbits = 0; p.lambda = 0.0f;   // no l2 term
+  p.spin_limit = 0;
+  p.seed_lo = p.seed_hi = p.step = 0;
 
-  int dev = 0, sms = 0, per_sm = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
-      cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, worker_absmax_kernel<false>, kThreads, 0) !=
-          cudaSuccess)
-    return QADAM_ERR_CUDA;
-  long long grid = (long long)sms * (per_sm > 0 ? per_sm : 1);
+  long long grid = setup.grid;
   if (grid > p.total_tiles) grid = p.total_tiles;
   worker_absmax_kernel<false><<<(int)grid, kThreads, 0, st>>>(p);
-  if (cudaGetLastError() != cudaSuccess) return QADAM_ERR_CUDA;
+  if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
   static_copy_scales_kernel<<<(n + 255) / 256, 256, 0, st>>>(acc, scales, n);
-  if (cudaGetLastError() != cudaSuccess) return QADAM_ERR_CUDA;
+  if (!cuda_ok(cudaGetLastError())) return QADAM_ERR_CUDA;
   return QADAM_OK;
 }

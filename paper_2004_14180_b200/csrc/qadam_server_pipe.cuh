@@ -4,11 +4,15 @@
 // One CTA per SM loops over 2048-element tiles.  A producer warp brings each
 // tile's inputs (x, m, v and the n workers' code runs of 512 or 768 bytes) into a ring of
 // shared-memory stages with bulk asynchronous copies that complete on an
-// mbarrier; two groups of eight consumer warps take alternate tiles, decode,
-// average and update in place in shared memory and write the packed broadcast; a
-// storer warp sends the updated x, m, v back with bulk stores and frees the stage.  Global-memory latency is covered by
-// the copies in flight (stages x tile bytes per SM), not by occupancy, so the
-// consumers keep their registers for arithmetic.
+// mbarrier; two groups of eight consumer warps take alternate tiles.  A consumer
+// warp first finds out which workers have anything but level 0 in its 256 codes
+// (one 16-byte load per lane covers a quarter of a worker's codes, a ballot gives
+// the answer for eight workers at once), decodes those in worker order, takes the
+// tile's x, m, v into registers and hands the stage back to the producer at once;
+// the update, the weight quantizer and the stores to global memory follow from
+// registers, while the stage is already being refilled.  Global-memory latency is
+// covered by the copies in flight (stages x tile bytes per SM), not by occupancy,
+// so the consumers keep their registers for arithmetic.
 //
 // Every wait on an mbarrier is bounded: when a wait runs out the thread raises a
 // CTA-wide abort flag and the TIMEOUT bit of the status word, every role leaves
@@ -22,16 +26,13 @@
 namespace qadam {
 
 constexpr int kPipeTile = 2048;                 // elements per pipeline tile
-#ifndef QADAM_PIPE_GROUPS
-#define QADAM_PIPE_GROUPS 2
-#endif
-constexpr int kPipeGroups = QADAM_PIPE_GROUPS;  // consumer groups; group g takes tiles g, g + groups, ...
+constexpr int kPipeGroups = 2;                  // consumer groups; group g takes tiles g, g + groups, ...
 constexpr int kPipeGroupThreads = 256;          // 8 warps per group, 8 elements per thread and tile
 constexpr int kPipeConsumers = kPipeGroups * kPipeGroupThreads;
-constexpr int kPipeThreads = kPipeConsumers + 64;   // + producer warp + storer warp
+constexpr int kPipeThreads = kPipeConsumers + 32;   // + producer warp
 constexpr int kPipeMaxWorkers = 64;
-constexpr int kPipeMaxStages = 8;
-constexpr unsigned kSpinLimit = 1u << 22;
+constexpr int kPipeMaxStages = 16;
+constexpr unsigned kSpinLimit = 1u << 22;       // default bound on the polls of one wait
 
 __device__ __forceinline__ unsigned smem_u32(const void* p) {
   return (unsigned)__cvta_generic_to_shared(p);
@@ -99,11 +100,12 @@ __device__ __forceinline__ void fence_async_shared() {
   asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
 }
 
-// Waits for the phase with the given parity; gives up after kSpinLimit polls or
+// Waits for the phase with the given parity; gives up after `limit` polls or
 // as soon as another thread has raised the abort flag.
 __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsigned parity,
-                                                  volatile int* abort_flag, unsigned* status) {
-  for (unsigned it = 0; it < kSpinLimit; ++it) {
+                                                  volatile int* abort_flag, unsigned* status,
+                                                  unsigned limit) {
+  for (unsigned it = 0; it < limit; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if (it >= 32) {
       if (*abort_flag) return false;
@@ -158,8 +160,7 @@ __host__ __device__ inline int pipe_legal_stages(int stages) {
 
 struct PipeSmem {
   unsigned long long full[kPipeMaxStages];      // producer -> consumers (bytes landed, header and scales written)
-  unsigned long long computed[kPipeMaxStages];  // consumers -> storer
-  unsigned long long empty[kPipeMaxStages];     // storer -> producer
+  unsigned long long empty[kPipeMaxStages];     // consumers -> producer (the stage has been read out)
   int abort_flag;
 };
 
@@ -299,10 +300,27 @@ __device__ __forceinline__ unsigned opaque_u32(unsigned v) {
   return r;
 }
 
-// Bytes ahead of the stage ring: the barriers and, for the table decode, 256 level values.
-__host__ __device__ inline size_t pipe_head_bytes(bool table_decode) {
-  return 256 + (table_decode ? 256 * sizeof(float) : 0);
+// Bytes ahead of the stage ring: the barriers, for the table decode 256 level values, and a
+// copy of the whole [n][S] table of scales when that is small (the producer then never waits
+// for global memory when a tile opens a new segment; 0 bytes: it reads the scales from global
+// memory whenever the segment changes).
+constexpr int kPipeBarrierBytes = 512;
+constexpr size_t kPipeScaleCacheMax = 16 * 1024;
+static_assert(sizeof(PipeSmem) <= kPipeBarrierBytes, "head of the shared-memory layout");
+__host__ __device__ inline size_t pipe_scale_cache_bytes(int n, int S) {
+  const size_t b = ((size_t)n * (size_t)S * sizeof(float) + 127) / 128 * 128;
+  return b <= kPipeScaleCacheMax ? b : 0;
 }
+__host__ __device__ inline size_t pipe_head_bytes(bool table_decode, size_t scale_cache_bytes) {
+  return kPipeBarrierBytes + (table_decode ? 256 * sizeof(float) : 0) + scale_cache_bytes;
+}
+
+
+// Slots of the liveness vote.  A warp's codes of one worker are two windows (the tile's two
+// 1024-element rows) of 16 * gb bytes, i.e. gb pieces of 16 bytes each; a worker gets
+// 2 * P slots, P the next power of two >= gb, so that a ballot holds a whole number of
+// workers.  Slot (row, piece) of worker i is lane-slot i * 2P + row * P + piece.
+__host__ __device__ constexpr int vote_pieces_pow2(int gb) { return gb <= 2 ? 2 : gb <= 4 ? 4 : 8; }
 
 // NW > 0: the worker count, known at compile time (the decode loop is unrolled and
 // every shared-memory offset is an immediate).  NW = 0: p.n workers, run-time loop.
@@ -312,12 +330,13 @@ template <bool SERVER_MOMENTS, int NW, int GB>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap codes_map,
                    const Tile* __restrict__ ptiles, const int num_ptiles, const int stages,
-                   const int inv_n_exact, const int skip_16ths) {
+                   const int inv_n_exact, const int scale_cache_bytes) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   PipeSmem* ps = reinterpret_cast<PipeSmem*>(smem_raw);
   static_assert(GB == 0 || GB == 2 || GB == 3, "code widths of the pipelined decode");
-  unsigned char* stage_base = smem_raw + pipe_head_bytes(GB == 0);
-  float* s_lut = reinterpret_cast<float*>(smem_raw + 256);      // table decode only
+  unsigned char* stage_base = smem_raw + pipe_head_bytes(GB == 0, (size_t)scale_cache_bytes);
+  float* s_lut = reinterpret_cast<float*>(smem_raw + kPipeBarrierBytes);      // table decode only
+  float* s_all_scales = reinterpret_cast<float*>(smem_raw + pipe_head_bytes(GB == 0, 0));   // [n][S], if cached
   const int n = NW > 0 ? NW : p.n;
   const int gb = GB > 0 ? GB : p.gbits;
   const unsigned stage_bytes = (unsigned)pipe_stage_bytes(n, SERVER_MOMENTS, gb);
@@ -328,6 +347,7 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
   const unsigned scales_off = kCodesOff + (unsigned)n * kRunBytes;
   const int tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
+  const unsigned spin = p.spin_limit;
 
   if constexpr (GB == 0) {
     // signed level value of every code (code = level index + L); codes past 2L never occur
@@ -341,11 +361,14 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
       s_lut[c] = q < 0 ? -lv : lv;
     }
   }
+  if (scale_cache_bytes > 0) {
+    const int total = n * p.S;
+    for (int idx = tid; idx < total; idx += kPipeThreads) s_all_scales[idx] = p.scales[idx];
+  }
   if (tid == 0) {
     for (int s = 0; s < stages; ++s) {
       mbar_init(&ps->full[s], 1);
-      mbar_init(&ps->computed[s], kPipeGroupThreads / 32);
-      mbar_init(&ps->empty[s], 1);
+      mbar_init(&ps->empty[s], kPipeGroupThreads / 32);
     }
     ps->abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -365,15 +388,33 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
     int s = 0;
     unsigned ph = 0;
     int issued = 0;
-    Tile t = my_tiles > 0 ? ptiles[blockIdx.x] : Tile{0, 0, 0};
+    // Tile descriptors are fetched 32 at a time, one per lane, a batch ahead of their use,
+    // and handed round by shuffles: the loop never waits for global memory.
+    auto fetch_batch = [&](int j0) -> Tile {
+      const int jj = j0 + lane;
+      return jj < my_tiles ? ptiles[blockIdx.x + (long long)jj * gridDim.x] : Tile{0, 0, 0};
+    };
+    Tile batch = fetch_batch(0);
+    Tile batch_next = fetch_batch(32);
     for (int j = 0; j < my_tiles; ++j) {
-      // next tile's descriptor is fetched while this one is issued
-      Tile tn = t;
-      if (j + 1 < my_tiles) tn = ptiles[blockIdx.x + (long long)(j + 1) * gridDim.x];
+      const int jl = j & 31;
+      if (jl == 0 && j > 0) {
+        batch = batch_next;
+        batch_next = fetch_batch(j + 32);
+      }
+      Tile t;
+      t.off = __shfl_sync(0xffffffffu, batch.off, jl);
+      t.count = __shfl_sync(0xffffffffu, batch.count, jl);
+      t.seg = __shfl_sync(0xffffffffu, batch.seg, jl);
       if (t.seg != cur_seg) {
         cur_seg = t.seg;
-        if (lane < n) sc0 = p.scales[(long long)lane * p.S + t.seg];
-        if (lane + 32 < n) sc1 = p.scales[(long long)(lane + 32) * p.S + t.seg];
+        if (scale_cache_bytes > 0) {
+          if (lane < n) sc0 = s_all_scales[lane * p.S + t.seg];
+          if (lane + 32 < n) sc1 = s_all_scales[(lane + 32) * p.S + t.seg];
+        } else {
+          if (lane < n) sc0 = p.scales[(long long)lane * p.S + t.seg];
+          if (lane + 32 < n) sc1 = p.scales[(long long)(lane + 32) * p.S + t.seg];
+        }
         if (GB == 3) {
           // half of a scale below 2^-120 may fall between floats; such a segment is summed
           // with a rounded product instead of a fused one
@@ -384,7 +425,7 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
       }
       // a fresh barrier passes a wait on the parity opposite to its first phase
       bool ok = true;
-      if (lane == 0) ok = mbar_wait_bounded(&ps->empty[s], ph ^ 1u, abort_flag, p.status);
+      if (lane == 0) ok = mbar_wait_bounded(&ps->empty[s], ph ^ 1u, abort_flag, p.status, spin);
       ok = __shfl_sync(0xffffffffu, ok, 0);
       if (!ok) break;
       unsigned char* st = stage_base + (size_t)s * stage_bytes;
@@ -410,13 +451,13 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
           bulk_load(sx + kPipeTile, p.m + t.off, fbytes, &ps->full[s]);
           bulk_load(sx + 2 * kPipeTile, p.v + t.off, fbytes, &ps->full[s]);
         }
-        // coordinate in words of the map: 32-bit (GB > 0) or 64-bit (table decode)
+        // coordinate in words of the map: 32-bit (GB > 0) or 64-bit (table decode); the host
+        // only selects this kernel when the last tile's coordinate fits an int
         const int c0 = GB > 0 ? (int)(t.off >> 5) * GB : (int)(t.off >> 6) * gb;
         tensor_load_2d(st + kCodesOff, &codes_map, c0, 0, &ps->full[s]);
       }
       ++issued;
       if (++s == stages) { s = 0; ph ^= 1u; }
-      t = tn;
     }
     // drain after an abort: nothing may still be landing in shared memory when the CTA exits
     __syncwarp();
@@ -432,37 +473,11 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
         }
       }
     }
-  } else if (warp == kPipeConsumers / 32 + 1) {
-    // ------------------------------------------------------------------ storer
-    int s = 0;
-    unsigned ph = 0;
-    for (int j = 0; j < my_tiles; ++j) {
-      bool ok = true;
-      if (lane == 0) ok = mbar_wait_bounded(&ps->computed[s], ph, abort_flag, p.status);
-      ok = __shfl_sync(0xffffffffu, ok, 0);
-      if (!ok) break;
-      if (lane == 0) {
-        unsigned char* st = stage_base + (size_t)s * stage_bytes;
-        const StageHeader hd = *reinterpret_cast<const StageHeader*>(st);
-        float* sx = reinterpret_cast<float*>(st + kStageHeaderBytes);
-        const unsigned fbytes = (unsigned)hd.count * 4u;
-        bulk_store(p.x + hd.off, sx, fbytes);
-        if (SERVER_MOMENTS) {
-          bulk_store(p.m + hd.off, sx + kPipeTile, fbytes);
-          bulk_store(p.v + hd.off, sx + 2 * kPipeTile, fbytes);
-        }
-        bulk_commit();
-        bulk_wait_read_all();                    // the stage has been read out
-        mbar_arrive(&ps->empty[s]);
-      }
-      if (++s == stages) { s = 0; ph ^= 1u; }
-    }
-    if (lane == 0) bulk_wait_all();               // writes are complete before the kernel ends
   } else {
     // ------------------------------------------------------------------ consumers
     // Two groups of 8 warps take alternate tiles, so that one group computes while
-    // the other waits for its data or hands its tile to the storer.  In a tile a
-    // thread owns elements 4t..4t+3 of both 1024-element rows.
+    // the other waits for its data.  In a tile a thread owns elements 4t..4t+3 of both
+    // 1024-element rows.
     const int group = tid / kPipeGroupThreads;
     const int gt = tid - group * kPipeGroupThreads;           // 0..255
     const int gwarp = gt >> 5;
@@ -482,40 +497,54 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
     const int tb_next = tb_word + 1 < 4 * gb ? tb_word + 1 : tb_word;
     const int tb_shift = (4 * gb * lane) & 31;
     const unsigned tb_cmask = (1u << gb) - 1u;
-    const unsigned tb_fmask = gb == 8 ? 0xffffffffu : (1u << (4 * gb)) - 1u;
-    unsigned tb_zero = 0;                                    // four level-0 codes
-    for (int c = 0; c < 4; ++c) tb_zero |= (unsigned)p.L << (c * gb);
-    bool sparse_mode = true;          // warp-uniform: look for workers with nothing but level 0
-    int dense_tiles_left = 0;
-    int dense_span = 8;
+
+    // Liveness vote.  With a max-abs scale most codes are level 0, and a worker whose 256
+    // codes in this warp's two rows are all level 0 adds +0 to every sum, which changes
+    // nothing (a sum is never -0).  Each lane compares one 16-byte piece of one worker's
+    // window with the pattern of level-0 codes; a ballot then tells, for 32 / kSlots workers
+    // at once, which have anything to add, and only those are decoded, in increasing worker
+    // order (the order of the sum is unchanged).
+    const int v_p2 = vote_pieces_pow2(gb);
+    const int v_slots = 2 * v_p2;                             // per worker
+    const int sl_log = v_slots == 4 ? 2 : v_slots == 8 ? 3 : 4;
+    const int v_slot = lane & (v_slots - 1);
+    const int v_row = v_slot >= v_p2 ? 1 : 0;
+    const int v_piece = v_slot & (v_p2 - 1);
+    const bool v_piece_ok = v_piece < gb;
+    const int v_worker0 = lane >> sl_log;                     // worker of this lane in ballot 0
+    const int v_per_ballot = 32 >> sl_log;                    // workers per ballot
+    const int v_off = v_row * kRowBytes + v_piece * 16 + gwarp * 16 * gb;
+    const unsigned v_gmask = v_slots == 4 ? 0xfu : v_slots == 8 ? 0xffu : 0xffffu;
+    // level-0 codes (code L) as they sit in the four words of the lane's piece: the window
+    // starts on a code boundary, so word j of it is the endless repetition of L in fields of
+    // gb bits, read from bit 32 j on
+    unsigned kz[4];
+    {
+      unsigned long long rep = (unsigned long long)p.L;
+      for (int width = gb; width < 64; width *= 2) rep |= rep << width;
+#pragma unroll
+      for (int t = 0; t < 4; ++t) kz[t] = (unsigned)(rep >> ((32 * (4 * v_piece + t)) % gb));
+    }
+
     for (int j = 0; j < my_tiles; ++j) {
       if (j % kPipeGroups == group) {
         // every lane waits for itself; the warp then agrees on the outcome so that it never splits
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->full[s], ph, abort_flag, p.status))) break;
+        if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->full[s], ph, abort_flag, p.status, spin))) break;
         unsigned char* st = stage_base + (size_t)s * stage_bytes;
         const StageHeader hd = *reinterpret_cast<const StageHeader*>(st);
         const bool act0 = gt * 4 < hd.count;                   // warp-uniform
         const bool act1 = kPipeTile / 2 + gt * 4 < hd.count;
+        float2 a[4];
+        float4 x4[2], m4[2], v4[2];
         if (act0) {
-          float* sx = reinterpret_cast<float*>(st + kStageHeaderBytes) + gt * 4;
           // ternary: the thread's byte of a row; five levels: the first of its two bytes
           // (table decode: the first byte of the warp's packed row)
           const unsigned char* s_codes =
               st + kCodesOff + (GB == 2 ? gt : GB == 3 ? gwarp * 48 + ((lane * 3) >> 1) : gwarp * 16 * gb);
           const bool tiny = GB == 3 && hd.tiny != 0;
           const float2* s_scale = reinterpret_cast<const float2*>(st + scales_off);
-          float2 a[4];
 #pragma unroll
           for (int c = 0; c < 4; ++c) a[c] = make_float2(0.0f, 0.0f);
-          // Zero skipping.  With a max-abs scale most codes are level 0 (ternary: code 1,
-          // byte 0x55 for four of them; five levels: code 2), and a worker whose 256 codes
-          // in this warp's two rows are all level 0 adds +0 to every sum, which changes
-          // nothing (a sum is never -0).  The warp first votes, worker by worker and without branching, on
-          // whether any lane holds a code other than 1, then decodes only the workers that
-          // do, in increasing worker order (the order of the sum is unchanged).  When
-          // more than an eighth of the workers have something to add the warp stops
-          // looking for a while: the votes cost about half a decode, so denser codes are
-          // decoded faster without them.
           auto window = [&](int i, int r) -> unsigned {       // 3-bit codes: the lane's 16-bit window
             const unsigned char* q = s_codes + i * kRunBytes + r * kRowBytes;
             return (unsigned)q[0] | ((unsigned)q[1] << 8);
@@ -546,83 +575,72 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
               table_accumulate(s_scale[i].x, field(i, 0), field(i, 1));
             }
           };
-          auto contribute_pair = [&](int i0, int i1, bool two) {
-            const float2 sc0 = s_scale[i0];
-            const float2 sc1 = two ? s_scale[i1] : make_float2(0.0f, 0.0f);
-            if constexpr (GB == 2) {
-              const unsigned p0 = s_codes[i0 * kRunBytes], p1 = s_codes[i0 * kRunBytes + kRowBytes];
-              const unsigned q0 = s_codes[i1 * kRunBytes], q1 = s_codes[i1 * kRunBytes + kRowBytes];
-              decode_accumulate(sc0, p0, p1, k01, k23, mg, a);
-              decode_accumulate(sc1, q0, q1, k01, k23, mg, a);
-            } else if constexpr (GB == 0) {
-              const unsigned p0 = field(i0, 0), p1 = field(i0, 1);
-              const unsigned q0 = field(i1, 0), q1 = field(i1, 1);
-              table_accumulate(sc0.x, p0, p1);
-              table_accumulate(sc1.x, q0, q1);
-            } else {
-              const unsigned p0 = window(i0, 0), p1 = window(i0, 1);
-              const unsigned q0 = window(i1, 0), q1 = window(i1, 1);
-              decode_accumulate5<false>(sc0, p0, p1, fl, a);
-              decode_accumulate5<false>(sc1, q0, q1, fl, a);
+          // ballot b: one bit per slot of workers b * v_per_ballot ... ; a slot beyond the
+          // window's pieces or the last worker votes "nothing"
+          const unsigned char* v_base = st + kCodesOff + v_off;
+          auto vote = [&](int b) -> unsigned {
+            const int i = b * v_per_ballot + v_worker0;
+            bool nz = false;
+            if (v_piece_ok && i < n) {
+              const uint4 w = *reinterpret_cast<const uint4*>(v_base + i * kRunBytes);
+              nz = (((w.x ^ kz[0]) | (w.y ^ kz[1])) | ((w.z ^ kz[2]) | (w.w ^ kz[3]))) != 0u;
             }
+            return __ballot_sync(0xffffffffu, nz);
           };
-          auto has_nonzero = [&](int i) -> unsigned long long {
-            bool nz;
-            if constexpr (GB == 2) {
-              const unsigned b0 = s_codes[i * kRunBytes];
-              const unsigned b1 = s_codes[i * kRunBytes + kRowBytes];
-              nz = (b0 & b1 & 0x55u) != 0x55u;
-            } else if constexpr (GB == 0) {
-              nz = (((field(i, 0) ^ tb_zero) | (field(i, 1) ^ tb_zero)) & tb_fmask) != 0u;
-            } else {
-              nz = (((window(i, 0) ^ fl.zero) | (window(i, 1) ^ fl.zero)) & fl.field) != 0u;
+          auto decode_live = [&](int b, unsigned bal) {        // the live workers of one ballot, in order
+            while (bal) {
+              const int g = (__ffs((int)bal) - 1) >> sl_log;
+              bal &= ~(v_gmask << (g << sl_log));
+              contribute(b * v_per_ballot + g);
             }
-            return __any_sync(0xffffffffu, nz) ? 1ull : 0ull;
           };
           if (tiny) {
             // rare: every worker, products rounded before they are added
 #pragma unroll 1
             for (int i = 0; i < n; ++i)
               decode_accumulate5<true>(s_scale[i], window(i, 0), window(i, 1), fl, a);
-          } else if (sparse_mode) {
-            unsigned long long live = 0;
-            if constexpr (NW > 0) {
-#pragma unroll kUnroll
-              for (int i = 0; i < NW; ++i) live |= has_nonzero(i) << i;
-            } else {
-#pragma unroll 4
-              for (int i = 0; i < n; ++i) live |= has_nonzero(i) << i;
+          } else if constexpr (NW > 0 && GB > 0) {
+            constexpr int kBallots = (NW * 2 * vote_pieces_pow2(GB) + 31) / 32;
+            unsigned bal[kBallots];
+            int live = 0;
+#pragma unroll
+            for (int b = 0; b < kBallots; ++b) {
+              bal[b] = vote(b);
+              unsigned t = bal[b];                             // one bit per live worker
+              t |= t >> 1;
+              t |= t >> 2;
+              if (GB == 3) t |= t >> 4;
+              live += __popc(t & (GB == 2 ? 0x11111111u : 0x01010101u));
             }
-            if (16 * __popcll(live) > skip_16ths * n) {
-              // too many live workers for the vote to pay: decode everything for a while,
-              // looking again after 16, 32, ... up to 1024 tiles
-              sparse_mode = false;
-              dense_span = dense_span < 1024 ? 2 * dense_span : 1024;
-              dense_tiles_left = dense_span;
-            } else {
-              dense_span = 8;
-            }
-            // live workers two at a time, so that the loads and the bit work of one overlap
-            // the other's; an odd one out is paired with scale 0, which adds nothing
-            while (live) {
-              const int i0 = __ffsll((long long)live) - 1;
-              live &= live - 1;
-              const bool two = live != 0;
-              const int i1 = two ? __ffsll((long long)live) - 1 : i0;
-              live &= live - 1;
-              contribute_pair(i0, i1, two);
-            }
-          } else {
-            if constexpr (NW > 0) {
+            if (4 * live >= 3 * NW) {
+              // nearly every worker has something to add: the unrolled loop over all of them
 #pragma unroll kUnroll
               for (int i = 0; i < NW; ++i) contribute(i);
             } else {
-#pragma unroll 4
-              for (int i = 0; i < n; ++i) contribute(i);
+#pragma unroll
+              for (int b = 0; b < kBallots; ++b) decode_live(b, bal[b]);
             }
-            if (--dense_tiles_left <= 0) sparse_mode = true;
+          } else {
+            // run-time worker count or code width: ballots taken and served one at a time
+            const int nb = (n * v_slots + 31) >> 5;
+            for (int b = 0; b < nb; ++b) decode_live(b, vote(b));
           }
-          // pads beyond the tile's length decode whatever the stage held; they are not used
+          // the tile's state into registers; pads beyond the tile's length are not used
+          const float* sx = reinterpret_cast<const float*>(st + kStageHeaderBytes) + gt * 4;
+#pragma unroll
+          for (int r = 0; r < 2; ++r) {
+            if (r == 1 && !act1) break;
+            x4[r] = *reinterpret_cast<const float4*>(sx + r * (kPipeTile / 2));
+            if constexpr (SERVER_MOMENTS) {
+              m4[r] = *reinterpret_cast<const float4*>(sx + kPipeTile + r * (kPipeTile / 2));
+              v4[r] = *reinterpret_cast<const float4*>(sx + 2 * kPipeTile + r * (kPipeTile / 2));
+            }
+          }
+        }
+        // everything this warp needs of the stage is in registers: hand it back
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&ps->empty[s]);
+        if (act0) {
           float2 d[4];
           if (inv_n_exact) {
             const float2 inv = make_float2(p.inv_nf, p.inv_nf);
@@ -635,40 +653,30 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
 #pragma unroll
           for (int r = 0; r < 2; ++r) {
             if (r == 1 && !act1) break;
-            float* rx = sx + r * (kPipeTile / 2);
-            const float4 x4 = *reinterpret_cast<const float4*>(rx);
+            const long long e0 = hd.off + r * (kPipeTile / 2);
             float xx[4];
             if constexpr (SERVER_MOMENTS) {
-              float* rm = rx + kPipeTile;
-              float* rv = rx + 2 * kPipeTile;
-              const float4 m4 = *reinterpret_cast<const float4*>(rm);
-              const float4 v4 = *reinterpret_cast<const float4*>(rv);
-              float2 m01 = make_float2(m4.x, m4.y), m23 = make_float2(m4.z, m4.w);
-              float2 v01 = make_float2(v4.x, v4.y), v23 = make_float2(v4.z, v4.w);
+              float2 m01 = make_float2(m4[r].x, m4[r].y), m23 = make_float2(m4[r].z, m4[r].w);
+              float2 v01 = make_float2(v4[r].x, v4[r].y), v23 = make_float2(v4[r].z, v4[r].w);
               moments2(p.h, d[2 * r], m01, v01);
               moments2(p.h, d[2 * r + 1], m23, v23);
-              xx[0] = __fsub_rn(x4.x, adam_step(p.h, m01.x, v01.x, p.alpha));
-              xx[1] = __fsub_rn(x4.y, adam_step(p.h, m01.y, v01.y, p.alpha));
-              xx[2] = __fsub_rn(x4.z, adam_step(p.h, m23.x, v23.x, p.alpha));
-              xx[3] = __fsub_rn(x4.w, adam_step(p.h, m23.y, v23.y, p.alpha));
-              *reinterpret_cast<float4*>(rm) = make_float4(m01.x, m01.y, m23.x, m23.y);
-              *reinterpret_cast<float4*>(rv) = make_float4(v01.x, v01.y, v23.x, v23.y);
+              xx[0] = __fsub_rn(x4[r].x, adam_step(p.h, m01.x, v01.x, p.alpha));
+              xx[1] = __fsub_rn(x4[r].y, adam_step(p.h, m01.y, v01.y, p.alpha));
+              xx[2] = __fsub_rn(x4[r].z, adam_step(p.h, m23.x, v23.x, p.alpha));
+              xx[3] = __fsub_rn(x4[r].w, adam_step(p.h, m23.y, v23.y, p.alpha));
+              st_f4(p.m + e0 + gt * 4, make_float4(m01.x, m01.y, m23.x, m23.y));
+              st_f4(p.v + e0 + gt * 4, make_float4(v01.x, v01.y, v23.x, v23.y));
             } else {
-              xx[0] = __fsub_rn(x4.x, d[2 * r].x);
-              xx[1] = __fsub_rn(x4.y, d[2 * r].y);
-              xx[2] = __fsub_rn(x4.z, d[2 * r + 1].x);
-              xx[3] = __fsub_rn(x4.w, d[2 * r + 1].y);
+              xx[0] = __fsub_rn(x4[r].x, d[2 * r].x);
+              xx[1] = __fsub_rn(x4[r].y, d[2 * r].y);
+              xx[2] = __fsub_rn(x4[r].z, d[2 * r + 1].x);
+              xx[3] = __fsub_rn(x4[r].w, d[2 * r + 1].y);
             }
-            *reinterpret_cast<float4*>(rx) = make_float4(xx[0], xx[1], xx[2], xx[3]);
-            if (p.kx >= 0) {
-              const long long e0 = hd.off + r * (kPipeTile / 2);
+            st_f4(p.x + e0 + gt * 4, make_float4(xx[0], xx[1], xx[2], xx[3]));
+            if (p.kx >= 0)
               broadcast_row(xx, p.kx, p.xbits, p.wcodes, p.wresid, e0 + gt * 4, e0 + gwarp * 128, lane);
-            }
           }
         }
-        fence_async_shared();                              // my writes, before the storer's bulk reads
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&ps->computed[s]);
       }
       if (++s == stages) { s = 0; ph ^= 1u; }
     }

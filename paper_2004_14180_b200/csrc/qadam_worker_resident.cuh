@@ -43,7 +43,6 @@
 
 namespace qadam {
 
-constexpr unsigned kWSpinLimit = 1u << 21;     // polls of a pair record before giving up
 
 __device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
   unsigned v;
@@ -156,6 +155,8 @@ worker_resident_kernel(const WorkerResidentParams rp) {
   const int warp = tid >> 5, lane = tid & 31;
   const int cta = (int)blockIdx.x, ctas = (int)gridDim.x;
   const int estages = rp.estages;
+  const unsigned spin = p.spin_limit;                           // polls of one wait before giving up
+  const unsigned pair_spin = spin > 1u ? spin >> 1 : 1u;        // polls of a pair's record
 
   if (tid == 0) {
     for (int s = 0; s < estages; ++s) {
@@ -199,8 +200,8 @@ worker_resident_kernel(const WorkerResidentParams rp) {
       if (lane == 0) {
         // the slot must have been read out by the store side (a fresh barrier passes a wait on
         // the parity opposite to its first phase), the ring stage by the consumers
-        ok = mbar_wait_bounded(&ps->slot_free[slot], slot_ph ^ 1u, abort_flag, p.status) &&
-             mbar_wait_bounded(&ps->e_empty[s], ph ^ 1u, abort_flag, p.status);
+        ok = mbar_wait_bounded(&ps->slot_free[slot], slot_ph ^ 1u, abort_flag, p.status, spin) &&
+             mbar_wait_bounded(&ps->e_empty[s], ph ^ 1u, abort_flag, p.status, spin);
         if (ok) {
           RLoadHeader* hd = &ps->load_hd[i & (kRHeaders - 1)];
           hd->pair = (long long)worker * p.S + cur.seg;
@@ -254,7 +255,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
     if (lane == 0) {
       for (long long i = 0; i < my_tiles; ++i) {
         const int hi = (int)(i & (kRHeaders - 1));
-        if (!mbar_wait_bounded(&ps->hd_ready[hi], (unsigned)(i / kRHeaders) & 1u, abort_flag, p.status)) break;
+        if (!mbar_wait_bounded(&ps->hd_ready[hi], (unsigned)(i / kRHeaders) & 1u, abort_flag, p.status, spin)) break;
         const RLoadHeader hd = ps->load_hd[hi];
         acc_max = max(acc_max, hd.max_bits);
         acc_cnt += 1;
@@ -301,7 +302,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
             const int kmax = cur.need < ctas ? cur.need : ctas;
             const unsigned long long* w = rp.words + pair * ctas;
             unsigned mx = 0;
-            for (unsigned it = 0; it < kWSpinLimit; ++it) {
+            for (unsigned it = 0; it < pair_spin; ++it) {
               unsigned cnt = 0;
               mx = 0;
               for (int k = lane; k < kmax; k += 32) {
@@ -314,7 +315,9 @@ worker_resident_kernel(const WorkerResidentParams rp) {
               cnt = __reduce_add_sync(0xffffffffu, cnt);
               mx = __reduce_max_sync(0xffffffffu, mx);
               if (cnt >= (unsigned)cur.need) { ok = true; break; }
-              if (*abort_flag) break;
+              // the flag is raised by other warps at any moment: the lanes must agree on
+              // what they saw, or some would leave while the rest wait in the next reduction
+              if (__any_sync(0xffffffffu, *abort_flag != 0)) break;
               __nanosleep(it < 64 ? 40 : 400);
             }
             __threadfence_block();                       // the words, before u is read out of the slots
@@ -325,7 +328,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
             }
           } else {
             if (lane == 0) {
-              for (unsigned it = 0; it < kWSpinLimit; ++it) {
+              for (unsigned it = 0; it < pair_spin; ++it) {
                 if (ld_acquire_u32(rp.done + pair) >= (unsigned)cur.need) { ok = true; break; }
                 if (*abort_flag) break;
                 __nanosleep(it < 64 ? 40 : 400);
@@ -348,7 +351,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
           ready_pair = pair;
         }
         if (lane == 0) {
-          ok = mbar_wait_bounded(&ps->cmd_empty[cs], cph ^ 1u, abort_flag, p.status);
+          ok = mbar_wait_bounded(&ps->cmd_empty[cs], cph ^ 1u, abort_flag, p.status, spin);
           if (ok) {
             RCommand* cd = &ps->cmd[cs];
             cd->off = cur.off;
@@ -407,7 +410,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
         step_j();
         if (i + 2 < my_tiles) ahead = rp.rtiles[pj];                 // descriptor of tile i + 2
       }
-      if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->e_full[s], ph, abort_flag, p.status))) break;
+      if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->e_full[s], ph, abort_flag, p.status, spin))) break;
       RLoadHeader* hdp = &ps->load_hd[i & (kRHeaders - 1)];
       const int slot = hdp->slot, count = hdp->count;
       float* su = reinterpret_cast<float*>(slot_base + (size_t)slot * kRSlotBytes) + gt * 4;
@@ -497,7 +500,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
     int cs = 0;
     unsigned cph = 0;
     for (long long i = 0; i < my_tiles; ++i) {
-      if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->cmd_full[cs], cph, abort_flag, p.status))) break;
+      if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->cmd_full[cs], cph, abort_flag, p.status, spin))) break;
       const RCommand cd = ps->cmd[cs];
       const float* su = reinterpret_cast<const float*>(slot_base + (size_t)cd.slot * kRSlotBytes) + gt * 4;
       // u into registers; from here on neither the slot nor the command is needed
@@ -513,7 +516,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
         mbar_arrive(&ps->slot_free[cd.slot]);
         mbar_arrive(&ps->cmd_empty[cs]);
       }
-      const float sc = __uint_as_float(cd.scale_bits);
+      const GradScale gs = grad_scale<MODE>(__uint_as_float(cd.scale_bits), p.k);
       unsigned char* cw = p.gcodes + (long long)cd.worker * p.gcode_bytes;
       float* ew = p.e + (long long)cd.worker * p.D + cd.off + gt * 4;
 #pragma unroll
@@ -524,7 +527,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
         unsigned code[4];
         float en[4];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) code[c] = quantize_grad<MODE>(uu[c], sc, p.k, p.L, en[c]);
+        for (int c = 0; c < 4; ++c) code[c] = quantize_grad<MODE>(uu[c], gs, p.k, p.L, en[c]);
         *reinterpret_cast<float4*>(ew + q * kRowElems) = make_float4(en[0], en[1], en[2], en[3]);
         const long long row_elem = cd.off + q * kRowElems + gwarp * 128;
         void* dst = cw + row_elem * p.bits / 8;

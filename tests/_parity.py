@@ -30,13 +30,14 @@ class Pair:
     """One problem held twice: `gpu` (qb.QAdam) and `cpu` (oracle.OracleState)."""
 
     def __init__(self, seg_len, n, kg, kx, placement, x1=None, grid_g=0, beta1=0.9, beta2=0.999,
-                 eps=1e-8, lr=1e-3, want_wresid=False):
+                 eps=1e-8, lr=1e-3, want_wresid=False, options=None, seed=0):
         self.lr = lr
         x1_t = None if x1 is None else torch.as_tensor(x1, dtype=torch.float32)
         self.gpu = qb.QAdam(seg_len, n, kg=kg, kx=kx, placement=placement, beta1=beta1, beta2=beta2,
-                            eps=eps, lr=lr, grid_g=grid_g, x1=x1_t, want_wresid=want_wresid)
+                            eps=eps, lr=lr, grid_g=grid_g, x1=x1_t, want_wresid=want_wresid,
+                            options=options, seed=seed)
         self.cpu = oracle.OracleState(seg_len, n, kg, kx, placement, beta1, beta2, eps,
-                                      grid_g=grid_g, want_wresid=want_wresid)
+                                      grid_g=grid_g, want_wresid=want_wresid, seed=seed)
         if x1 is not None:
             self.cpu.set_weights(np.asarray(x1, dtype=np.float32))
         else:

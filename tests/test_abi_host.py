@@ -36,7 +36,7 @@ def test_library_exports_every_declared_function(lib):
 
 def _cfg(**kw):
     base = dict(d=1000, n=2, num_segments=1, seg_len=None, kg=0, kx=0, grid_g=0, placement=0,
-                beta1=0.9, beta2=0.999, eps=1e-8, lr=1e-3, stream=None)
+                beta1=0.9, beta2=0.999, eps=1e-8, lr=1e-3, stream=None, seed=0)
     base.update(kw)
     return qb.QAdamConfig(**base)
 
@@ -67,7 +67,8 @@ def test_code_widths(lib):
 @pytest.mark.parametrize("kw,code", [
     (dict(d=0), -2), (dict(n=0), -2), (dict(num_segments=0), -2),
     (dict(num_segments=3), -1),                      # seg_len NULL with S > 1
-    (dict(kg=-2), -3), (dict(kg=15), -3), (dict(kg=7, grid_g=1), -3), (dict(grid_g=2), -3),
+    (dict(kg=-2), -3), (dict(kg=15), -3), (dict(kg=7, grid_g=1), -3), (dict(grid_g=3), -3),
+    (dict(kg=1, grid_g=2), -3), (dict(kg=-1, grid_g=2), -3),      # the stochastic operator is ternary only
     (dict(kx=15), -3), (dict(kx=-2), -3),
     (dict(placement=2), -10),
     (dict(beta1=1.0), -8), (dict(beta2=-0.1), -8), (dict(eps=0.0), -8), (dict(lr=float("nan")), -8),
@@ -94,6 +95,41 @@ def test_null_arguments(lib):
     assert lib.qadam_server_step(None, 1, C.c_float(0.1)) == -1
     assert lib.qadam_destroy(None) == -1
     assert qb.qadam_strerror(-6) == "step out of order"
+
+
+def test_options_are_checked_before_anything_else_happens(lib):
+    # unknown enumerators, a negative test hook and non-zero reserved fields: QADAM_ERR_SIZE,
+    # decided on the host before any CUDA call (so this runs without a GPU)
+    cfg, bufs, ctx = _cfg(), qb.QAdamBuffers(), C.c_void_p()
+    bad = [qb.QAdamOptions(server_kernel=2), qb.QAdamOptions(worker_kernel=5), qb.QAdamOptions(hand_over=-1),
+           qb.QAdamOptions(test_missing_tiles=-3)]
+    r = qb.QAdamOptions()
+    r.reserved[1] = 1
+    bad.append(r)
+    for opt in bad:
+        assert lib.qadam_create_ex(C.byref(cfg), C.byref(bufs), C.byref(opt), C.byref(ctx)) == -2
+        assert not ctx.value
+    assert lib.qadam_create_ex(None, C.byref(bufs), None, C.byref(ctx)) == -1
+    # valid options, missing buffers: the next check in line answers
+    assert lib.qadam_create_ex(C.byref(cfg), C.byref(bufs), C.byref(qb.QAdamOptions()), C.byref(ctx)) == -1
+
+
+def test_range_and_shard_calls_reject_bad_arguments(lib):
+    assert lib.qadam_server_step_range(None, 1, C.c_float(0.1), 0, 128) == -1
+    assert lib.qadam_finish_step(None, 1) == -1
+    cuts = (C.c_int64 * 3)()
+    assert lib.qadam_shard_cuts(None, 2, cuts) == -1
+    assert lib.qadam_shard_cuts(C.byref(_cfg()), 0, cuts) == -2
+    assert lib.qadam_shard_cuts(C.byref(_cfg(d=0)), 2, cuts) == -2
+    assert lib.qadam_shard_cuts(C.byref(_cfg(d=10000)), 2, cuts) == 0
+    assert list(cuts) == [0, 8192, 10112]          # tiles of 4096; D = 10000 padded to 10112
+
+
+def test_stochastic_operator_sizes(lib):
+    sz = qb.qadam_query_sizes(_cfg(grid_g=qb.GRID_STOCHASTIC))
+    assert sz["gcode_bytes"] == sz["D"] // 4       # ternary codes
+    assert qb.qadam_grad_code_bits(0, qb.GRID_STOCHASTIC) == 2
+    assert qb.qadam_grad_code_bits(1, qb.GRID_STOCHASTIC) < 0
 
 
 def test_layout_agrees_with_the_oracle(lib, oracle):

@@ -23,11 +23,11 @@ def _rand_grads(rng, n, d, sigma=0.01):
 
 
 def _run(seg, n, kg, kx, placement, T=3, grid=0, seed=0, sigma=0.01, wresid=False, x_sigma=0.2,
-         split=False, **hyper):
+         split=False, options=None, **hyper):
     rng = np.random.default_rng(seed)
     d = sum(seg)
     x1 = (rng.standard_normal(d) * x_sigma).astype(np.float32)
-    p = Pair(seg, n, kg, kx, placement, x1=x1, grid_g=grid, want_wresid=wresid, **hyper)
+    p = Pair(seg, n, kg, kx, placement, x1=x1, grid_g=grid, want_wresid=wresid, options=options, **hyper)
     p.compare_state()                        # first broadcast Q_x(x_1)
     for t in range(T):
         p.step(_rand_grads(rng, n, d, sigma), split_workers=split and t % 2 == 1)
@@ -284,27 +284,28 @@ def test_on_chip_worker_l2_term_many_tiles(kx, placement):
 
 
 @pytest.mark.parametrize("placement", [S_MODE, W_MODE])
-def test_on_chip_worker_counter_hand_over(placement, monkeypatch):
+def test_on_chip_worker_counter_hand_over(placement):
     # the on-chip kernel hands a pair's scale over through one word per (pair, CTA) while the
-    # workspace has room for them, else through one counter per pair; QADAM_RESIDENT_COUNTERS
-    # (read at every call) forces the second route
-    monkeypatch.setenv("QADAM_RESIDENT_COUNTERS", "1")
+    # workspace has room for them, else through one counter per pair; the hand_over option
+    # forces the second route
+    import paper_2004_14180_b200 as qb
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     seg = [sms * 2 * 4096 + 300, 5000, 64, 70000, 129]
-    _run(seg, 3, 0, 0, placement, T=3, seed=90 + placement)
+    _run(seg, 3, 0, 0, placement, T=3, seed=90 + placement,
+         options=qb.QAdamOptions(hand_over=qb.HANDOVER_COUNTERS))
 
 
 @pytest.mark.parametrize("placement", [S_MODE, W_MODE])
-def test_streaming_launches_only(placement, monkeypatch):
-    # QADAM_WORKER_KERNEL=split (read when the context is created) sends every pair through
-    # the two streaming launches, the route that otherwise only pairs too large for the chip,
-    # partial worker ranges and some l2 cases take
-    monkeypatch.setenv("QADAM_WORKER_KERNEL", "split")
+def test_streaming_launches_only(placement):
+    # worker_kernel = STREAMING sends every pair through the two streaming launches, the
+    # route that otherwise only pairs too large for the chip, partial worker ranges and some
+    # l2 cases take
+    import paper_2004_14180_b200 as qb
     rng = np.random.default_rng(70 + placement)
     seg = [9000, 64, 129, 3 * 4096 + 640, 1, 70000]
     n, d = 4, sum([9000, 64, 129, 3 * 4096 + 640, 1, 70000])
     x1 = (rng.standard_normal(d) * 0.2).astype(np.float32)
-    p = Pair(seg, n, 0, 1, placement, x1=x1)
+    p = Pair(seg, n, 0, 1, placement, x1=x1, options=qb.QAdamOptions(worker_kernel=qb.WORKER_STREAMING))
     one, two = p.gpu.worker_pass_model()
     assert one == 0 and two == n * p.gpu.D
     for t in range(3):
@@ -405,3 +406,110 @@ def test_config_resnet18_shaped_paper_placement_and_single_scale():
     w = qi.get_workload("resnet18_qg_qx_k0")
     _run_workload(w, 3, W_MODE)
     _run_workload(w.with_(per_tensor_scale=False), 3, S_MODE)
+
+
+def test_config_resnet18_shaped_all_steps():
+    """The ResNet-18-shaped workload over its full T = 100 steps (gradient and weight
+    quantizers on, moments on the server): codes and scales compared after every step, the
+    whole state every tenth step and at the end.  Gradients are drawn on the GPU."""
+    w = qi.get_workload("resnet18_qg_qx_k0")
+    dev = torch.device("cuda")
+    x1 = qi.initial_weights(w, "cpu").numpy()
+    p = Pair(w.scale_seg_len, w.n, w.kg, w.kx, S_MODE, x1=x1, beta1=w.beta1, beta2=w.beta2, eps=w.eps, lr=w.lr)
+    for t in range(1, w.steps + 1):
+        g = torch.stack([qi.gradients(w, t, i, dev) for i in range(w.n)]).cpu().numpy()
+        p.step(g, threads=8)
+        if t % 10 == 0:
+            p.compare_state()
+    assert p.step_no == 100
+    p.close()
+
+
+# ---------------------------------------------------------------- the plain server kernel
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+@pytest.mark.parametrize("kg,grid", [(0, 0), (1, 0), (3, 0), (3, 1)])
+@pytest.mark.parametrize("n", [65, 128])
+def test_plain_server_kernel_many_workers(n, kg, grid, placement):
+    """More than 64 workers go through the grid-stride server kernel (its own ternary decode
+    and its per-worker table of level values for the other grids): several tiles, a ragged
+    tail, two segments with different scales."""
+    _run([3 * 4096 + 640, 130, 4096], n, kg, 1, placement, T=2, grid=grid, seed=700 + n + 10 * kg + grid)
+
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+@pytest.mark.parametrize("kg", [0, 1, 3])
+def test_plain_server_kernel_sparse_and_dense_regions(kg, placement):
+    # the same kernel chosen by option at a worker count the pipelined pass would take,
+    # over a vector with a dense third and a sparse rest
+    import paper_2004_14180_b200 as qb
+    rng = np.random.default_rng(80 + kg)
+    d, n = 1 << 21, 6
+    dense_end = d * 3 // 10
+    x1 = (rng.standard_normal(d) * 0.05).astype(np.float32)
+    p = Pair([d], n, kg, 0, placement, x1=x1, options=qb.QAdamOptions(server_kernel=qb.SERVER_PLAIN))
+    for t in range(2):
+        g = (rng.standard_normal((n, d)) * 1e-4).astype(np.float32)
+        g[:, :dense_end] = rng.standard_normal((n, dense_end)).astype(np.float32)
+        hits = rng.integers(dense_end, d, (n, 300))
+        for i in range(n):
+            g[i, hits[i]] = rng.choice(np.array([4.0, -4.0, 2.0, -1.0], np.float32), 300)
+        g[:, d - 1] = 5.0
+        p.step(g, threads=4)
+        p.compare_state()
+    p.close()
+
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+@pytest.mark.parametrize("density", [1e-4, 1e-3, 1e-2, 0.1])
+def test_pipelined_server_code_densities(density, placement):
+    """The pipelined pass decodes only the workers that have a non-zero code in a warp's 256
+    elements and switches to the unrolled loop over all workers when most do: densities on
+    both sides of that switch, n = 16 (compile-time worker count) and n = 5 (run-time)."""
+    rng = np.random.default_rng(int(density * 1e6) + placement)
+    d = 3 * (1 << 18) + 640
+    for n in (16, 5):
+        x1 = (rng.standard_normal(d) * 0.05).astype(np.float32)
+        p = Pair([d], n, 0, 0, placement, x1=x1)
+        for t in range(2):
+            g = (rng.standard_normal((n, d)) * 1e-6).astype(np.float32)
+            hit = rng.random((n, d)) < density
+            g[hit] = np.where(rng.random(int(hit.sum())) < 0.5, 1.0, -1.0).astype(np.float32)
+            g[:, 0] = 1.5
+            p.step(g, threads=4)
+            p.compare_state()
+        p.close()
+
+
+# ---------------------------------------------------------------- the stochastic ternary operator
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+@pytest.mark.parametrize("n,seed", [(3, 1), (16, (1 << 63) + 12345), (70, 20200429)])
+def test_stochastic_ternary_operator(n, seed, placement):
+    """The comparison operator of Section 5.1 (level 1 with probability |u| / max|u|): both
+    sides draw their coins from Philox4x32-10 with counter (element / 4, worker, step) and key
+    = seed, so codes are bit-identical; several tiles, ragged tails, partial worker calls,
+    the pipelined and the plain server pass, with the l2 term switched on for one step."""
+    rng = np.random.default_rng(900 + n)
+    seg = [3 * 4096 + 640, 130, 70000, 1]
+    d = sum(seg)
+    x1 = (rng.standard_normal(d) * 0.2).astype(np.float32)
+    p = Pair(seg, n, 0, 1, placement, x1=x1, grid_g=2, seed=seed)
+    assert p.gpu.worker_pass_model()[0] == 0          # this operator runs in the streaming launches
+    lam = [0.0, 0.0, 5e-4, 0.0]
+    for t in range(4):
+        p.set_regularization(lam[t])
+        p.step(_rand_grads(rng, n, d), split_workers=t == 1)
+        p.compare_state()
+    live = np.mean(p.cpu.gcodes != 0x55)
+    assert live > 0.2                                  # far denser than the deterministic ternary codes
+    p.close()
+
+
+def test_stochastic_operator_is_ternary_only():
+    import paper_2004_14180_b200 as qb
+    with pytest.raises(qb.QAdamError) as ei:
+        qb.QAdam([1000], 2, kg=1, grid_g=qb.GRID_STOCHASTIC)
+    assert ei.value.code == -3
+    with pytest.raises(qb.QAdamError):
+        qb.QAdam([1000], 2, kg=-1, grid_g=qb.GRID_STOCHASTIC)
