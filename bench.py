@@ -81,6 +81,9 @@ def parse_args():
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--mode", default="replicas", choices=["replicas", "ps"],
+                    help="with several GPUs: independent replicas (default), or ONE problem with the "
+                         "workers dealt out to the ranks and the server sharded (codes exchanged over NCCL)")
     ap.add_argument("--no-configs", action="store_true",
                     help="skip the per-configuration records (key `configs` of the line)")
     ap.add_argument("--config-steps", type=int, default=5)
@@ -524,10 +527,88 @@ def run_b200(args):
         dist.destroy_process_group()
 
 
+def run_ps(args):
+    """One problem over all ranks: rank r compresses its share of the workers, the packed codes
+    are exchanged (all-to-all), each rank serves its range of the vector, and the packed weights
+    are gathered back.  Total work is fixed as ranks are added: strong scaling."""
+    import torch
+    import torch.distributed as dist
+    import qadam_inputs as qi
+    import paper_2004_14180_b200 as qb
+    from paper_2004_14180_b200 import ps
+
+    rank, world, local = rank_env()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py --mode ps needs a CUDA device")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if not dist.is_initialized():
+        if world == 1:
+            os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+            os.environ.setdefault("MASTER_PORT", "29511")
+        dist.init_process_group("nccl", rank=rank, world_size=world, device_id=dev)
+    w = get_workload(args)
+    if w.n % world:
+        w = w.with_(n=(w.n + world - 1) // world * world)        # workers are dealt out evenly
+    placement = qb.PLACE_SERVER if args.placement == "server" else qb.PLACE_WORKER
+    x1 = qi.initial_weights(w, dev)
+    q = qb.QAdam(w.scale_seg_len, w.n, kg=w.kg, kx=w.kx, placement=placement, beta1=w.beta1,
+                 beta2=w.beta2, eps=w.eps, lr=w.lr, x1=x1, device=dev)
+    q.set_regularization(args.weight_decay)
+    del x1
+    drv = ps.ShardedStep(q, always_communicate=True)
+    k = drv.plan.workers_per_rank
+    g = torch.zeros(k, q.D, dtype=torch.float32, device=dev)
+    for j, i in enumerate(drv.plan.workers_of(rank)):
+        g[j].copy_(q.to_padded(qi.gradients(w, 1, i, dev)))
+
+    def sync_all():
+        torch.cuda.synchronize()
+        dist.barrier()
+        torch.cuda.synchronize()
+
+    step = 0
+    for _ in range(max(3, args.warmup)):
+        step += 1
+        drv.step(step, g)
+    sync_all()
+    launches0 = q.launches
+    clocks = ClockSampler(local)
+    time.sleep(0.25)
+    sync_all()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        step += 1
+        drv.step(step, g)
+    e1.record()
+    sync_all()
+    ms_step = max_over_ranks(e0.elapsed_time(e1), world, dev) / args.steps
+    clock_info = clocks.stop()
+    status = q.poll_status()
+    if rank == 0:
+        wire = ps.wire_bytes_per_step(drv.plan, q.S)
+        cfg = workload_config(w, args, extra={
+            "parallelism": f"sharded parameter server over {world} rank(s): {k} worker(s) and 1/{world} of the "
+                           "vector per rank; all-to-all of packed codes, all-gather of scales, broadcast of "
+                           "the packed weights (NCCL)",
+            "D_padded": q.D, "wire_bytes_per_step": wire, "shard_cuts": list(drv.plan.cuts)})
+        line = {"metric": METRIC, "value": w.d * w.n / (ms_step * 1e-3), "unit": UNIT, "n_gpus": world,
+                "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms_step,
+                "higher_is_better": True, "scaling": "strong", "vs_baseline": None, "dtype": "f32",
+                "data": "synthetic", "mode": "ps", "config": cfg, "clocks": clock_info,
+                "gpu_launches": int(q.launches - launches0), "device_status": int(status)}
+        print(json.dumps(line), flush=True)
+    q.close()
+    dist.destroy_process_group()
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         run_reference(args)
+    elif args.mode == "ps":
+        run_ps(args)
     else:
         run_b200(args)
 

@@ -129,9 +129,9 @@ typedef struct {
  *                 memory, one CTA per SM) whenever the codes are at most 8 bits wide and
  *                 n <= 64, else the plain grid-stride kernel.  PLAIN: always the latter.
  *  worker_kernel  AUTO: (worker, segment) pairs that fit in the SMs' shared memory go
- *                 through one persistent kernel that reads g and e once; larger pairs and
- *                 calls for a part of the workers take two streaming launches (max-abs,
- *                 then quantize).  STREAMING: always the two launches.
+ *                 through one persistent kernel that reads g and e once; larger pairs take
+ *                 two streaming launches (max-abs, then quantize), and so does everything
+ *                 under the stochastic operator.  STREAMING: always the two launches.
  *  hand_over      how the persistent worker kernel passes a pair's scale between CTAs.
  *                 AUTO: one 64-bit word per (pair, CTA) while those fit in 32 MB of
  *                 workspace, else one counter per pair and atomics.  COUNTERS: always the
@@ -222,7 +222,8 @@ int qadam_server_step(qadam_ctx* ctx, int64_t step, float lr_t);
  * exactly as qadam_server_step serves them: the same sums in the same order, the same
  * bits in x, m, v, wcodes and wresid on that range; nothing outside it is read or
  * written (gcodes: bytes [elem_begin*b_g/8, elem_end*b_g/8) of each worker's stream, and
- * every worker's scales).  Both ends must be shard cuts (qadam_shard_cuts), else
+ * every worker's scales).  Both ends must be tile boundaries, such as the cuts that
+ * qadam_shard_cuts returns (any start of a 4096-element tile of a segment, or D), else
  * QADAM_ERR_SIZE.  The caller vouches that all n workers' codes of the range and all
  * scales are in gcodes / scales (compressed here or received from elsewhere): the check of
  * qadam_server_step on the workers compressed by THIS context does not apply.
@@ -319,7 +320,7 @@ int qadam_profile_enable(qadam_ctx* ctx, int enable);
 int qadam_profile_read(qadam_ctx* ctx, double* ms, int64_t* launches);
 
 /* Instrumentation: how the worker side of this context moves its data when all
- * workers are compressed in one call.  one_pass: padded (worker, element) pairs that
+ * workers are compressed.  one_pass: padded (worker, element) pairs that
  * belong to (worker, segment) pairs small enough to be held on chip between the
  * max-abs reduction and the quantization (read from HBM once); two_pass: pairs in
  * segments too large for that (read twice).  The sum is n * D. */

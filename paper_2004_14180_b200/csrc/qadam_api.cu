@@ -207,13 +207,13 @@ struct qadam_ctx {
   float lambda = 0.0f;       // l2 term (qadam_set_regularization)
   int pipe_stages = 0;
   size_t pipe_smem = 0;
-  int pipe_scale_cache = 0;  // bytes of the scales table the pipelined pass keeps in shared memory
+  bool pipe_wide = false;    // the pipelined pass walks the 4096-element tiles (four rows) instead of the 2048-element ones
   qadam_options opt = {};
   unsigned spin_limit = kSpinLimit;
   bool range_open = false;   // a range of the current step has been served (qadam_server_step_range)
   CUtensorMap codes_map;
   unsigned* d_done = nullptr;
-  // on-chip worker kernel (moments on the server, all workers in one call): grid > 0 when in use
+  // on-chip worker kernel: grid > 0 when in use
   int grid_resident = 0;
   int res_slots = 0, res_estages = 0;
   size_t res_smem = 0;
@@ -285,26 +285,33 @@ ServerKernel pick_server(const qadam_ctx* c) {
   }
 }
 
-using PipeKernel = void (*)(const ServerParams, const CUtensorMap, const Tile*, int, int, int, int);
+using PipeKernel = void (*)(const ServerParams, const CUtensorMap, const Tile*, int, int, int);
 
-template <bool SM, int GB>
+template <bool SM, int GB, int XB, int ROWS>
 PipeKernel pick_pipe_n(int n) {
   switch (n) {
-    case 4: return server_pipe_kernel<SM, 4, GB>;
-    case 8: return server_pipe_kernel<SM, 8, GB>;
-    case 16: return server_pipe_kernel<SM, 16, GB>;
-    case 32: return server_pipe_kernel<SM, 32, GB>;
-    default: return server_pipe_kernel<SM, 0, GB>;
+    case 4: return server_pipe_kernel<SM, 4, GB, XB, ROWS>;
+    case 8: return server_pipe_kernel<SM, 8, GB, XB, ROWS>;
+    case 16: return server_pipe_kernel<SM, 16, GB, XB, ROWS>;
+    case 32: return server_pipe_kernel<SM, 32, GB, XB, ROWS>;
+    default: return server_pipe_kernel<SM, 0, GB, XB, ROWS>;
   }
 }
 
 PipeKernel pick_pipe(const qadam_ctx* c) {
   const bool sm = c->cfg.placement == QADAM_PLACE_SERVER;
-  if (c->geo.gmode == G_FIVE) return sm ? pick_pipe_n<true, 3>(c->cfg.n) : pick_pipe_n<false, 3>(c->cfg.n);
-  if (c->geo.gmode == G_TERNARY || c->geo.gmode == G_STOCHASTIC)
-    return sm ? pick_pipe_n<true, 2>(c->cfg.n) : pick_pipe_n<false, 2>(c->cfg.n);
+  const int n = c->cfg.n;
+  if (c->geo.gmode == G_FIVE) return sm ? pick_pipe_n<true, 3, 0, 2>(n) : pick_pipe_n<false, 3, 0, 2>(n);
+  if (c->geo.gmode == G_TERNARY || c->geo.gmode == G_STOCHASTIC) {
+    // ternary gradient codes; ternary weights (kx = 0) have a path of their own; with the
+    // moments on the workers the pass is decode bound and takes tiles of four rows
+    if (c->pipe_wide)
+      return c->cfg.kx == 0 ? pick_pipe_n<false, 2, 2, 4>(n) : pick_pipe_n<false, 2, 0, 4>(n);
+    if (c->cfg.kx == 0) return sm ? pick_pipe_n<true, 2, 2, 2>(n) : pick_pipe_n<false, 2, 2, 2>(n);
+    return sm ? pick_pipe_n<true, 2, 0, 2>(n) : pick_pipe_n<false, 2, 0, 2>(n);
+  }
   // any other grid of at most 8 bits: table decode, worker count at run time
-  return sm ? server_pipe_kernel<true, 0, 0> : server_pipe_kernel<false, 0, 0>;
+  return sm ? server_pipe_kernel<true, 0, 0, 0, 2> : server_pipe_kernel<false, 0, 0, 0, 2>;
 }
 
 using WorkerResidentKernel = void (*)(const WorkerResidentParams);
@@ -514,20 +521,27 @@ int qadam_create_ex(const qadam_config* cfg, const qadam_buffers* b, const qadam
     const bool table = c->geo.gmode == G_POW2 || c->geo.gmode == G_UNIFORM;
     const bool pipe_codes = c->geo.gmode == G_TERNARY || c->geo.gmode == G_STOCHASTIC || c->geo.gmode == G_FIVE ||
                             (table && c->geo.gbits <= 8);
-    const size_t sb = pipe_stage_bytes(cfg->n, sm_mom, pipe_codes ? c->geo.gbits : 2);
-    const size_t scale_cache = pipe_scale_cache_bytes(cfg->n, cfg->num_segments);
-    const size_t head = pipe_head_bytes(table, scale_cache);
+    const size_t head = pipe_head_bytes(table);
     const bool want_plain = o.server_kernel == QADAM_SERVER_PLAIN;
-    int stages = (int)(((size_t)max_smem - head) / sb);
-    stages = pipe_legal_stages(std::min(stages, kPipeMaxStages));
+    auto stages_for = [&](int tile_elems) {
+      const size_t sb = pipe_stage_bytes(cfg->n, sm_mom, pipe_codes ? c->geo.gbits : 2, tile_elems);
+      return pipe_legal_stages(std::min((int)(((size_t)max_smem - head) / sb), kPipeMaxStages));
+    };
+    // With the moments on the workers the quantized quantity is Adam's normalised update,
+    // whose codes are dense, and the pass is bound by the decode, not by memory: tiles of four
+    // rows give a thread twice the independent work per tile, as long as four stages still fit.
+    const bool ternary_codes = c->geo.gmode == G_TERNARY || c->geo.gmode == G_STOCHASTIC;
+    c->pipe_wide = !sm_mom && ternary_codes && stages_for(kPipeWideTile) >= 4;
+    const int tile_elems = c->pipe_wide ? kPipeWideTile : kPipeTile;
+    const size_t sb = pipe_stage_bytes(cfg->n, sm_mom, pipe_codes ? c->geo.gbits : 2, tile_elems);
+    int stages = stages_for(tile_elems);
     // the tensor copy addresses a tile's codes by a 32-bit coordinate in words of the stream
     // (32-bit words, 64-bit for the table decode): longer streams take the plain kernel
     const bool coord_fits = (long long)c->geo.gcode_bytes / (table ? 8 : 4) < (1ll << 31);
     if (!want_plain && pipe_codes && coord_fits && cfg->n <= kPipeMaxWorkers && stages >= 2 &&
         make_codes_tensor_map(&c->codes_map, b->gcodes, (long long)c->geo.gcode_bytes, cfg->n,
-                              c->geo.gbits, table)) {
+                              c->geo.gbits, table, tile_elems)) {
       c->pipe_stages = stages;
-      c->pipe_scale_cache = (int)scale_cache;
       c->pipe_smem = head + (size_t)stages * sb;
       if (!cuda_ok(cudaFuncSetAttribute(pick_pipe(c), cudaFuncAttributeMaxDynamicSharedMemorySize,
                                         (int)c->pipe_smem))) {
@@ -538,7 +552,7 @@ int qadam_create_ex(const qadam_config* cfg, const qadam_buffers* b, const qadam
   if (!plan_worker_grids(c)) { delete c; return QADAM_ERR_CUDA; }
   c->grid_server = resident_grid(sk, c->server_smem, c->sm_count);
   c->grid_bcast = resident_grid(weight_broadcast_kernel, 0, c->sm_count);
-  // Worker side, all workers in one call.  Segments small enough to be held by the
+  // Worker side.  Segments small enough to be held by the
   // on-chip kernel (u stays in shared memory between the
   // max-abs reduction and the quantization, so g and e are read once) go through that
   // kernel; larger segments need two passes over memory whatever is done and take the two
@@ -683,9 +697,9 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
     if (!cuda_ok(cudaMemsetAsync(p.scale_bits + (size_t)worker_begin * p.S, 0,
                                  sizeof(unsigned) * (size_t)worker_count * p.S, c->stream)))
       return QADAM_ERR_CUDA;
-    bool on_chip = c->grid_resident > 0 && worker_begin == 0 && worker_count == c->cfg.n && !l2_split(c);
+    bool on_chip = c->grid_resident > 0 && !l2_split(c);
     if (on_chip) {
-      const size_t pairs = (size_t)c->cfg.n * p.S;
+      const size_t pairs = (size_t)c->cfg.n * p.S;     // all pairs' records are cleared, the call's are used
       const bool l2 = c->lambda != 0.0f;
       const bool use_words = !l2 && c->d_words != nullptr && c->grid_resident <= kWordCtas &&
                              c->opt.hand_over == QADAM_HANDOVER_AUTO;
@@ -699,7 +713,7 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
       rp.rtiles = c->d_rtiles;
       rp.done = c->d_done;
       rp.TR = (int)c->geo.rtiles.size();
-      rp.total = (long long)c->cfg.n * rp.TR;
+      rp.total = (long long)worker_count * rp.TR;
       rp.slots = c->res_slots;
       rp.estages = c->res_estages;
       void* args[] = {&rp};
@@ -778,10 +792,12 @@ int launch_server(qadam_ctx* c, float alpha, long long tb, long long te, long lo
     if (c->pipe_stages > 0) {
       const int n = c->cfg.n;
       const int inv_exact = (n & (n - 1)) == 0 ? 1 : 0;
-      const int np = (int)(pe - pb);
+      // the walk is over the 2048-element tiles, or over the 4096-element ones (four rows)
+      const Tile* table = c->pipe_wide ? c->d_tiles + tb : c->d_ptiles + pb;
+      const int np = (int)(c->pipe_wide ? te - tb : pe - pb);
       const int pgrid = std::min(c->sm_count, np);
-      pick_pipe(c)<<<pgrid, kPipeThreads, c->pipe_smem, c->stream>>>(p, c->codes_map, c->d_ptiles + pb, np,
-                                                                      c->pipe_stages, inv_exact, c->pipe_scale_cache);
+      pick_pipe(c)<<<pgrid, kPipeThreads, c->pipe_smem, c->stream>>>(p, c->codes_map, table, np,
+                                                                      c->pipe_stages, inv_exact);
     } else {
       p.tiles = c->d_tiles + tb;
       p.tiles_per_worker = (int)(te - tb);

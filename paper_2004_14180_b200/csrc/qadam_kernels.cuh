@@ -50,7 +50,8 @@ __device__ __forceinline__ void held_fetch8(const WorkerParams& p, long long row
   const int F = 4 * p.xbits;                            // bits per lane = words per row
   const int w = (F * lane) >> 5;
   lo = __ldg(words + w);
-  hi = __ldg(words + (w + 1 < F ? w + 1 : w));
+  // the lane's field runs into the next word only for widths that do not divide 32
+  hi = ((F * lane) & 31) + F > 32 ? __ldg(words + w + 1) : 0u;
 }
 // ... and their values: (code - 2^kx) times the grid step, exact.
 __device__ __forceinline__ void held_decode8(const WorkerParams& p, int lane, unsigned lo, unsigned hi,
@@ -104,11 +105,42 @@ __device__ __forceinline__ void held_weights4(const WorkerParams& p, long long r
     out[2 * h + 1] = value((f >> p.xbits) & mask);
   }
 }
+// The held weights of a thread's 4 elements of a row as they are loaded when the weights are
+// packed codes of at most 8 bits: the two words that hold the lane's 4 codes, fetched together
+// with the loads of g and e and decoded when the row is processed.  Unquantized weights and
+// wider codes are read at the point of use (fetched stays false).
+struct HeldRaw {
+  unsigned lo, hi;
+  bool fetched;
+};
+__device__ __forceinline__ HeldRaw held_fetch(const WorkerParams& p, long long row_elem, int lane) {
+  HeldRaw h;
+  h.lo = h.hi = 0u;
+  h.fetched = p.kx >= 0 && p.xbits <= 8;
+  if (h.fetched) held_fetch8(p, row_elem, lane, h.lo, h.hi);
+  return h;
+}
+// g + lambda * (held weights) from what held_fetch loaded
+__device__ __forceinline__ void add_l2_term_held(const WorkerParams& p, long long row_elem, int lane,
+                                                 const HeldRaw& h, float gg[4]);
+
 // g + lambda * (held weights), each operation rounded once (Section 5.1's l2 term)
 __device__ __forceinline__ void add_l2_term(const WorkerParams& p, long long row_elem, int lane,
                                             float gg[4]) {
   float w[4];
   held_weights4(p, row_elem, lane, w);
+#pragma unroll
+  for (int c = 0; c < 4; ++c) gg[c] = __fadd_rn(gg[c], __fmul_rn(p.lambda, w[c]));
+}
+
+__device__ __forceinline__ void add_l2_term_held(const WorkerParams& p, long long row_elem, int lane,
+                                                 const HeldRaw& h, float gg[4]) {
+  if (!h.fetched) {
+    add_l2_term(p, row_elem, lane, gg);
+    return;
+  }
+  float w[4];
+  held_decode8(p, lane, h.lo, h.hi, w);
 #pragma unroll
   for (int c = 0; c < 4; ++c) gg[c] = __fadd_rn(gg[c], __fmul_rn(p.lambda, w[c]));
 }
@@ -180,7 +212,7 @@ __device__ __forceinline__ unsigned block_max(unsigned v, unsigned* smem8) {
 // or Inf ends up as the maximum and is reported by phase 2).
 // ---------------------------------------------------------------------------
 template <bool WORKER_MOMENTS, bool L2 = false>
-__global__ void __launch_bounds__(kThreads, WORKER_MOMENTS ? 2 : 4)
+__global__ void __launch_bounds__(kThreads, WORKER_MOMENTS ? 2 : (L2 ? 3 : 4))
 worker_absmax_kernel(const WorkerParams p) {
   __shared__ unsigned red[kThreads / 32];
   unsigned mx = 0;
@@ -201,6 +233,7 @@ worker_absmax_kernel(const WorkerParams p) {
     const float* gp = p.g + (long long)wl * p.D + tile.off;
     const long long so = (long long)w * p.D + tile.off;
     float4 gv[kRows], ev[kRows], mv[kRows], vv[kRows];
+    HeldRaw hw[L2 ? kRows : 1];
     bool act[kRows];
 #pragma unroll
     for (int r = 0; r < kRows; ++r) {
@@ -213,6 +246,8 @@ worker_absmax_kernel(const WorkerParams p) {
           mv[r] = ld_f4(p.m + so + idx);
           vv[r] = ld_f4(p.v + so + idx);
         }
+        if constexpr (L2)
+          hw[r] = held_fetch(p, tile.off + r * kRowElems + (threadIdx.x >> 5) * 128, threadIdx.x & 31);
       }
     }
 #pragma unroll
@@ -223,7 +258,7 @@ worker_absmax_kernel(const WorkerParams p) {
       float ee[4] = {ev[r].x, ev[r].y, ev[r].z, ev[r].w};
       float uu[4];
       if constexpr (L2)
-        add_l2_term(p, tile.off + r * kRowElems + (threadIdx.x >> 5) * 128, threadIdx.x & 31, gg);
+        add_l2_term_held(p, tile.off + r * kRowElems + (threadIdx.x >> 5) * 128, threadIdx.x & 31, hw[r], gg);
       if constexpr (WORKER_MOMENTS) {
         float mm[4] = {mv[r].x, mv[r].y, mv[r].z, mv[r].w};
         float vs[4] = {vv[r].x, vv[r].y, vv[r].z, vv[r].w};
@@ -257,14 +292,15 @@ template <bool U_IN_E, int MODE, bool L2 = false>
 __global__ void __launch_bounds__(kThreads)
 worker_quantize_kernel(const WorkerParams p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  // With u left in e's slot a tile brings only one array in, so two tiles are taken per
-  // round to keep as many loads in flight as the two-array form has.
-  constexpr int kPerRound = U_IN_E ? 2 : 1;
+  // Tiles per round of loads, then of arithmetic and stores.  (Two per round when only e is
+  // read, to have as many loads in flight as the two-array form, was measured slower.)
+  constexpr int kPerRound = 1;
   for (long long t0 = blockIdx.x; t0 < p.total_tiles; t0 += (long long)kPerRound * gridDim.x) {
     Tile tile[kPerRound];
     int wl[kPerRound];
     bool have[kPerRound];
     float4 gv[kPerRound][kRows], ev[kPerRound][kRows];
+    HeldRaw hw[kPerRound][L2 ? kRows : 1];
 #pragma unroll
     for (int a = 0; a < kPerRound; ++a) {
       const long long t = t0 + (long long)a * gridDim.x;
@@ -280,6 +316,8 @@ worker_quantize_kernel(const WorkerParams p) {
         if (idx < tile[a].count) {
           if constexpr (!U_IN_E) gv[a][r] = ld_f4_stream(gp + idx);
           ev[a][r] = ld_f4(p.e + so + idx);
+          if constexpr (L2 && !U_IN_E)
+            hw[a][r] = held_fetch(p, tile[a].off + r * kRowElems + warp * 128, lane);
         }
       }
     }
@@ -304,7 +342,7 @@ worker_quantize_kernel(const WorkerParams p) {
           for (int c = 0; c < 4; ++c) uu[c] = ee[c];
         } else {
           float gg[4] = {gv[a][r].x, gv[a][r].y, gv[a][r].z, gv[a][r].w};
-          if constexpr (L2) add_l2_term(p, tile[a].off + r * kRowElems + warp * 128, lane, gg);
+          if constexpr (L2) add_l2_term_held(p, tile[a].off + r * kRowElems + warp * 128, lane, hw[a][r], gg);
 #pragma unroll
           for (int c = 0; c < 4; ++c) uu[c] = __fadd_rn(gg[c], ee[c]);
         }

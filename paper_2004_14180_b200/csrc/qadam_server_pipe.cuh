@@ -25,7 +25,9 @@
 
 namespace qadam {
 
-constexpr int kPipeTile = 2048;                 // elements per pipeline tile
+constexpr int kPipeRowElems = 1024;             // a tile is 2 or 4 rows of 1024 elements (4 per consumer thread)
+constexpr int kPipeTile = 2 * kPipeRowElems;    // elements per pipeline tile (the default, two rows)
+constexpr int kPipeWideTile = 4 * kPipeRowElems;// four rows: decode-bound passes get more work per thread and tile
 constexpr int kPipeGroups = 2;                  // consumer groups; group g takes tiles g, g + groups, ...
 constexpr int kPipeGroupThreads = 256;          // 8 warps per group, 8 elements per thread and tile
 constexpr int kPipeConsumers = kPipeGroups * kPipeGroupThreads;
@@ -63,6 +65,21 @@ __device__ __forceinline__ bool mbar_try_wait(unsigned long long* bar, unsigned 
       : "memory");
   return ok != 0;
 }
+// The same, but the hardware may keep the thread suspended for up to `ns` nanoseconds while
+// the phase is incomplete (it resumes at once when the phase completes): a waiting warp then
+// takes no issue slots from the warps that have work.
+__device__ __forceinline__ bool mbar_try_wait_suspend(unsigned long long* bar, unsigned parity, unsigned ns) {
+  unsigned ok;
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+      "selp.u32 %0, 1, 0, p;\n\t}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity), "r"(ns)
+      : "memory");
+  return ok != 0;
+}
+constexpr unsigned kWaitSuspendNs = 1000;       // per poll; a wait gives up after `limit` polls
 // global -> shared, completion counted in bytes on `bar`
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gsrc, unsigned bytes,
                                           unsigned long long* bar) {
@@ -105,12 +122,10 @@ __device__ __forceinline__ void fence_async_shared() {
 __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsigned parity,
                                                   volatile int* abort_flag, unsigned* status,
                                                   unsigned limit) {
+  if (mbar_try_wait(bar, parity)) return true;
   for (unsigned it = 0; it < limit; ++it) {
-    if (mbar_try_wait(bar, parity)) return true;
-    if (it >= 32) {
-      if (*abort_flag) return false;
-      __nanosleep(100);
-    }
+    if (mbar_try_wait_suspend(bar, parity, kWaitSuspendNs)) return true;
+    if (*abort_flag) return false;
   }
   *abort_flag = 1;
   atomicOr(status, 2u);
@@ -125,7 +140,7 @@ __device__ __forceinline__ bool mbar_wait_bounded(unsigned long long* bar, unsig
 // wide: 64-bit words instead (a box side holds at most 256 elements, which 32-bit words
 // exceed from 5 bits per code on); coordinates and extents are then in 8-byte units.
 inline bool make_codes_tensor_map(CUtensorMap* map, const void* gcodes, long long gcode_bytes, int n,
-                                  int gbits, bool wide = false) {
+                                  int gbits, bool wide = false, int tile_elems = kPipeTile) {
   typedef CUresult (*EncodeTiled)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*,
                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
@@ -138,7 +153,7 @@ inline bool make_codes_tensor_map(CUtensorMap* map, const void* gcodes, long lon
   const int word = wide ? 8 : 4;
   const cuuint64_t dims[2] = {(cuuint64_t)(gcode_bytes / word), (cuuint64_t)n};
   const cuuint64_t strides[1] = {(cuuint64_t)gcode_bytes};          // bytes between rows
-  const cuuint32_t box[2] = {(cuuint32_t)(kPipeTile * gbits / (8 * word)), (cuuint32_t)n};
+  const cuuint32_t box[2] = {(cuuint32_t)(tile_elems * gbits / (8 * word)), (cuuint32_t)n};
   if (box[0] > 256 || box[1] > 256) return false;
   const cuuint32_t estr[2] = {1, 1};
   const CUresult r = reinterpret_cast<EncodeTiled>(fn)(
@@ -172,9 +187,10 @@ struct StageHeader {
 };
 constexpr int kStageHeaderBytes = 128;
 
-__host__ __device__ inline size_t pipe_stage_bytes(int n, bool server_moments, int gbits) {
-  const size_t state = (server_moments ? 3 : 1) * (size_t)kPipeTile * sizeof(float);
-  const size_t codes = (size_t)n * (kPipeTile * gbits / 8);
+__host__ __device__ inline size_t pipe_stage_bytes(int n, bool server_moments, int gbits,
+                                                   int tile_elems = kPipeTile) {
+  const size_t state = (server_moments ? 3 : 1) * (size_t)tile_elems * sizeof(float);
+  const size_t codes = (size_t)n * (tile_elems * gbits / 8);
   const size_t scales = ((size_t)n * 2 * sizeof(float) + 127) / 128 * 128;
   return kStageHeaderBytes + state + codes + scales;
 }
@@ -300,50 +316,70 @@ __device__ __forceinline__ unsigned opaque_u32(unsigned v) {
   return r;
 }
 
-// Bytes ahead of the stage ring: the barriers, for the table decode 256 level values, and a
-// copy of the whole [n][S] table of scales when that is small (the producer then never waits
-// for global memory when a tile opens a new segment; 0 bytes: it reads the scales from global
-// memory whenever the segment changes).
+// Bytes ahead of the stage ring: the barriers and, for the table decode, 256 level values.
 constexpr int kPipeBarrierBytes = 512;
-constexpr size_t kPipeScaleCacheMax = 16 * 1024;
 static_assert(sizeof(PipeSmem) <= kPipeBarrierBytes, "head of the shared-memory layout");
-__host__ __device__ inline size_t pipe_scale_cache_bytes(int n, int S) {
-  const size_t b = ((size_t)n * (size_t)S * sizeof(float) + 127) / 128 * 128;
-  return b <= kPipeScaleCacheMax ? b : 0;
-}
-__host__ __device__ inline size_t pipe_head_bytes(bool table_decode, size_t scale_cache_bytes) {
-  return kPipeBarrierBytes + (table_decode ? 256 * sizeof(float) : 0) + scale_cache_bytes;
+__host__ __device__ inline size_t pipe_head_bytes(bool table_decode) {
+  return kPipeBarrierBytes + (table_decode ? 256 * sizeof(float) : 0);
 }
 
-
-// Slots of the liveness vote.  A warp's codes of one worker are two windows (the tile's two
-// 1024-element rows) of 16 * gb bytes, i.e. gb pieces of 16 bytes each; a worker gets
-// 2 * P slots, P the next power of two >= gb, so that a ballot holds a whole number of
-// workers.  Slot (row, piece) of worker i is lane-slot i * 2P + row * P + piece.
+// Slots of the liveness vote.  A warp's codes of one worker are one window per row of the tile
+// (16 * gb bytes, i.e. gb pieces of 16 bytes each); a worker gets ROWS * P slots, P the next
+// power of two >= gb, so that a ballot holds a whole number of workers.  Slot (row, piece) of
+// worker i is lane-slot i * ROWS * P + row * P + piece.
 __host__ __device__ constexpr int vote_pieces_pow2(int gb) { return gb <= 2 ? 2 : gb <= 4 ? 4 : 8; }
+
+// Q_x for the grid {-1/2, 0, 1/2} (kx = 0) of 4 consecutive weights of one lane and the
+// packed store of the warp's row of 128 two-bit codes (32 bytes): the four codes of a lane
+// are one byte; two shuffle steps gather four lanes' bytes into a word, which lanes
+// 0, 4, ..., 28 store.  row_dst: address of the row's first code.
+__device__ __forceinline__ void broadcast_row_ternary(const float xx[4], unsigned char* row_dst,
+                                                      float* wresid_elem, int lane) {
+  unsigned field = 0;
+  float xq[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    // midpoint 1/4, ties toward zero; code = level index + 1
+    const bool up = xx[c] > 0.25f, down = xx[c] < -0.25f;
+    xq[c] = up ? 0.5f : (down ? -0.5f : 0.0f);
+    field |= (up ? 2u : (down ? 0u : 1u)) << (2 * c);
+  }
+  if (wresid_elem) {
+    st_f4(wresid_elem, make_float4(__fsub_rn(xx[0], xq[0]), __fsub_rn(xx[1], xq[1]),
+                                   __fsub_rn(xx[2], xq[2]), __fsub_rn(xx[3], xq[3])));
+  }
+  unsigned w = field | (__shfl_down_sync(0xffffffffu, field, 1) << 8);
+  w |= __shfl_down_sync(0xffffffffu, w, 2) << 16;
+  if ((lane & 3) == 0) reinterpret_cast<unsigned*>(row_dst)[lane >> 2] = w;
+}
 
 // NW > 0: the worker count, known at compile time (the decode loop is unrolled and
 // every shared-memory offset is an immediate).  NW = 0: p.n workers, run-time loop.
 // GB: bits per gradient code, 2 (ternary) or 3 (five levels); 0: any grid with p.gbits
 // (3..8) bits per code, decoded through a table of the signed level values.
-template <bool SERVER_MOMENTS, int NW, int GB>
+// XB: 2 when the weights are quantized to {-1/2, 0, 1/2} (kx = 0), which gets a path of its
+// own; 0: any p.kx, decided at run time.
+// ROWS: rows of 1024 elements per tile, 2 or 4 (a thread owns 4 elements of each row).
+template <bool SERVER_MOMENTS, int NW, int GB, int XB, int ROWS>
 __global__ void __launch_bounds__(kPipeThreads, 1)
 server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap codes_map,
                    const Tile* __restrict__ ptiles, const int num_ptiles, const int stages,
-                   const int inv_n_exact, const int scale_cache_bytes) {
+                   const int inv_n_exact) {
   extern __shared__ __align__(128) unsigned char smem_raw[];
   PipeSmem* ps = reinterpret_cast<PipeSmem*>(smem_raw);
   static_assert(GB == 0 || GB == 2 || GB == 3, "code widths of the pipelined decode");
-  unsigned char* stage_base = smem_raw + pipe_head_bytes(GB == 0, (size_t)scale_cache_bytes);
+  static_assert(XB == 0 || XB == 2, "weight code widths with a path of their own");
+  static_assert(ROWS == 2 || ROWS == 4, "rows per tile");
+  constexpr int kTile = ROWS * kPipeRowElems;
+  unsigned char* stage_base = smem_raw + pipe_head_bytes(GB == 0);
   float* s_lut = reinterpret_cast<float*>(smem_raw + kPipeBarrierBytes);      // table decode only
-  float* s_all_scales = reinterpret_cast<float*>(smem_raw + pipe_head_bytes(GB == 0, 0));   // [n][S], if cached
   const int n = NW > 0 ? NW : p.n;
   const int gb = GB > 0 ? GB : p.gbits;
-  const unsigned stage_bytes = (unsigned)pipe_stage_bytes(n, SERVER_MOMENTS, gb);
+  const unsigned stage_bytes = (unsigned)pipe_stage_bytes(n, SERVER_MOMENTS, gb, kTile);
   constexpr int kState = SERVER_MOMENTS ? 3 : 1;
-  constexpr unsigned kCodesOff = kStageHeaderBytes + kState * kPipeTile * 4;
-  const int kRunBytes = kPipeTile * gb / 8;              // one worker's codes of a tile
-  const int kRowBytes = kRunBytes / 2;                   // of one of its two 1024-element rows
+  constexpr unsigned kCodesOff = kStageHeaderBytes + kState * kTile * 4;
+  const int kRunBytes = kTile * gb / 8;                  // one worker's codes of a tile
+  const int kRowBytes = kRunBytes / ROWS;                // of one of its 1024-element rows
   const unsigned scales_off = kCodesOff + (unsigned)n * kRunBytes;
   const int tid = threadIdx.x;
   const int warp = tid >> 5, lane = tid & 31;
@@ -360,10 +396,6 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
                                : (p.gmode == G_FIVE ? level_value<G_FIVE>(a, p.k) : level_value<G_UNIFORM>(a, p.k));
       s_lut[c] = q < 0 ? -lv : lv;
     }
-  }
-  if (scale_cache_bytes > 0) {
-    const int total = n * p.S;
-    for (int idx = tid; idx < total; idx += kPipeThreads) s_all_scales[idx] = p.scales[idx];
   }
   if (tid == 0) {
     for (int s = 0; s < stages; ++s) {
@@ -388,33 +420,15 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
     int s = 0;
     unsigned ph = 0;
     int issued = 0;
-    // Tile descriptors are fetched 32 at a time, one per lane, a batch ahead of their use,
-    // and handed round by shuffles: the loop never waits for global memory.
-    auto fetch_batch = [&](int j0) -> Tile {
-      const int jj = j0 + lane;
-      return jj < my_tiles ? ptiles[blockIdx.x + (long long)jj * gridDim.x] : Tile{0, 0, 0};
-    };
-    Tile batch = fetch_batch(0);
-    Tile batch_next = fetch_batch(32);
+    Tile t = my_tiles > 0 ? ptiles[blockIdx.x] : Tile{0, 0, 0};
     for (int j = 0; j < my_tiles; ++j) {
-      const int jl = j & 31;
-      if (jl == 0 && j > 0) {
-        batch = batch_next;
-        batch_next = fetch_batch(j + 32);
-      }
-      Tile t;
-      t.off = __shfl_sync(0xffffffffu, batch.off, jl);
-      t.count = __shfl_sync(0xffffffffu, batch.count, jl);
-      t.seg = __shfl_sync(0xffffffffu, batch.seg, jl);
+      // next tile's descriptor is fetched while this one is issued
+      Tile tn = t;
+      if (j + 1 < my_tiles) tn = ptiles[blockIdx.x + (long long)(j + 1) * gridDim.x];
       if (t.seg != cur_seg) {
         cur_seg = t.seg;
-        if (scale_cache_bytes > 0) {
-          if (lane < n) sc0 = s_all_scales[lane * p.S + t.seg];
-          if (lane + 32 < n) sc1 = s_all_scales[(lane + 32) * p.S + t.seg];
-        } else {
-          if (lane < n) sc0 = p.scales[(long long)lane * p.S + t.seg];
-          if (lane + 32 < n) sc1 = p.scales[(long long)(lane + 32) * p.S + t.seg];
-        }
+        if (lane < n) sc0 = p.scales[(long long)lane * p.S + t.seg];
+        if (lane + 32 < n) sc1 = p.scales[(long long)(lane + 32) * p.S + t.seg];
         if (GB == 3) {
           // half of a scale below 2^-120 may fall between floats; such a segment is summed
           // with a rounded product instead of a fused one
@@ -439,7 +453,7 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
         hd->tiny = tiny;
       }
       __syncwarp();
-      // one elected lane issues the tile's four requests: x, m, v runs and the code box.
+      // one elected lane issues the tile's requests: x, m, v runs and the code box.
       // The box always carries n full rows of kRunBytes (beyond a short tile's length it holds
       // the neighbouring codes or zero fill, which nobody reads).
       if (lane == 0) {
@@ -448,8 +462,8 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
         float* sx = reinterpret_cast<float*>(st + kStageHeaderBytes);
         bulk_load(sx, p.x + t.off, fbytes, &ps->full[s]);
         if (SERVER_MOMENTS) {
-          bulk_load(sx + kPipeTile, p.m + t.off, fbytes, &ps->full[s]);
-          bulk_load(sx + 2 * kPipeTile, p.v + t.off, fbytes, &ps->full[s]);
+          bulk_load(sx + kTile, p.m + t.off, fbytes, &ps->full[s]);
+          bulk_load(sx + 2 * kTile, p.v + t.off, fbytes, &ps->full[s]);
         }
         // coordinate in words of the map: 32-bit (GB > 0) or 64-bit (table decode); the host
         // only selects this kernel when the last tile's coordinate fits an int
@@ -458,6 +472,7 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
       }
       ++issued;
       if (++s == stages) { s = 0; ph ^= 1u; }
+      t = tn;
     }
     // drain after an abort: nothing may still be landing in shared memory when the CTA exits
     __syncwarp();
@@ -476,13 +491,12 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
   } else {
     // ------------------------------------------------------------------ consumers
     // Two groups of 8 warps take alternate tiles, so that one group computes while
-    // the other waits for its data.  In a tile a thread owns elements 4t..4t+3 of both
-    // 1024-element rows.
+    // the other waits for its data.  In a tile a thread owns elements 4t..4t+3 of every
+    // 1024-element row.  The ring holds a multiple of the group count, so a group steps
+    // through its own stages only.
     const int group = tid / kPipeGroupThreads;
     const int gt = tid - group * kPipeGroupThreads;           // 0..255
     const int gwarp = gt >> 5;
-    int s = 0;
-    unsigned ph = 0;
     // -(2^E + 1) for the four code positions of a byte (E = 23, 21, 19, 17)
     const float2 k01 = make_float2(-(exp2i(23) + 1.0f), -(exp2i(21) + 1.0f));
     const float2 k23 = make_float2(-(exp2i(19) + 1.0f), -(exp2i(17) + 1.0f));
@@ -501,20 +515,20 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
     // Liveness vote.  With a max-abs scale most codes are level 0, and a worker whose 256
     // codes in this warp's two rows are all level 0 adds +0 to every sum, which changes
     // nothing (a sum is never -0).  Each lane compares one 16-byte piece of one worker's
-    // window with the pattern of level-0 codes; a ballot then tells, for 32 / kSlots workers
+    // window with the pattern of level-0 codes; a ballot then tells, for 32 / v_slots workers
     // at once, which have anything to add, and only those are decoded, in increasing worker
     // order (the order of the sum is unchanged).
     const int v_p2 = vote_pieces_pow2(gb);
-    const int v_slots = 2 * v_p2;                             // per worker
-    const int sl_log = v_slots == 4 ? 2 : v_slots == 8 ? 3 : 4;
+    const int v_slots = ROWS * v_p2;                          // per worker: 4, 8, 16 or 32
+    const int sl_log = v_slots == 4 ? 2 : v_slots == 8 ? 3 : v_slots == 16 ? 4 : 5;
     const int v_slot = lane & (v_slots - 1);
-    const int v_row = v_slot >= v_p2 ? 1 : 0;
+    const int v_row = v_slot / v_p2;
     const int v_piece = v_slot & (v_p2 - 1);
     const bool v_piece_ok = v_piece < gb;
     const int v_worker0 = lane >> sl_log;                     // worker of this lane in ballot 0
     const int v_per_ballot = 32 >> sl_log;                    // workers per ballot
     const int v_off = v_row * kRowBytes + v_piece * 16 + gwarp * 16 * gb;
-    const unsigned v_gmask = v_slots == 4 ? 0xfu : v_slots == 8 ? 0xffu : 0xffffu;
+    const unsigned v_gmask = v_slots == 4 ? 0xfu : v_slots == 8 ? 0xffu : v_slots == 16 ? 0xffffu : 0xffffffffu;
     // level-0 codes (code L) as they sit in the four words of the lane's piece: the window
     // starts on a code boundary, so word j of it is the endless repetition of L in fields of
     // gb bits, read from bit 32 j on
@@ -525,160 +539,233 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
 #pragma unroll
       for (int t = 0; t < 4; ++t) kz[t] = (unsigned)(rep >> ((32 * (4 * v_piece + t)) % gb));
     }
+    // per-thread pieces of the output addresses
+    float* const gx = p.x + gt * 4;
+    float* const gm = SERVER_MOMENTS ? p.m + gt * 4 : nullptr;
+    float* const gv = SERVER_MOMENTS ? p.v + gt * 4 : nullptr;
+    int dense_tiles_left = 0;         // warp-uniform: tiles for which the search for sparse structure is skipped
+    int dense_span = 8;
 
-    for (int j = 0; j < my_tiles; ++j) {
-      if (j % kPipeGroups == group) {
-        // every lane waits for itself; the warp then agrees on the outcome so that it never splits
-        if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->full[s], ph, abort_flag, p.status, spin))) break;
-        unsigned char* st = stage_base + (size_t)s * stage_bytes;
-        const StageHeader hd = *reinterpret_cast<const StageHeader*>(st);
-        const bool act0 = gt * 4 < hd.count;                   // warp-uniform
-        const bool act1 = kPipeTile / 2 + gt * 4 < hd.count;
-        float2 a[4];
-        float4 x4[2], m4[2], v4[2];
-        if (act0) {
-          // ternary: the thread's byte of a row; five levels: the first of its two bytes
-          // (table decode: the first byte of the warp's packed row)
-          const unsigned char* s_codes =
-              st + kCodesOff + (GB == 2 ? gt : GB == 3 ? gwarp * 48 + ((lane * 3) >> 1) : gwarp * 16 * gb);
-          const bool tiny = GB == 3 && hd.tiny != 0;
-          const float2* s_scale = reinterpret_cast<const float2*>(st + scales_off);
+    int s = group;
+    unsigned ph = 0;
+    for (int j = group; j < my_tiles; j += kPipeGroups) {
+      // every lane waits for itself; the warp then agrees on the outcome so that it never splits
+      if (!__all_sync(0xffffffffu, mbar_wait_bounded(&ps->full[s], ph, abort_flag, p.status, spin))) break;
+      unsigned char* st = stage_base + (size_t)s * stage_bytes;
+      const StageHeader hd = *reinterpret_cast<const StageHeader*>(st);
+      const bool act0 = gt * 4 < hd.count;                   // warp-uniform
+      auto active = [&](int r) { return r * kPipeRowElems + gt * 4 < hd.count; };   // monotone in r
+      float2 a[2 * ROWS];
+      float4 x4[ROWS], m4[ROWS], v4[ROWS];
+      if (act0) {
+        // ternary: the thread's byte of a row; five levels: the first of its two bytes
+        // (table decode: the first byte of the warp's packed row)
+        const unsigned char* s_codes =
+            st + kCodesOff + (GB == 2 ? gt : GB == 3 ? gwarp * 48 + ((lane * 3) >> 1) : gwarp * 16 * gb);
+        const bool tiny = GB == 3 && hd.tiny != 0;
+        const float2* s_scale = reinterpret_cast<const float2*>(st + scales_off);
 #pragma unroll
-          for (int c = 0; c < 4; ++c) a[c] = make_float2(0.0f, 0.0f);
-          auto window = [&](int i, int r) -> unsigned {       // 3-bit codes: the lane's 16-bit window
-            const unsigned char* q = s_codes + i * kRunBytes + r * kRowBytes;
-            return (unsigned)q[0] | ((unsigned)q[1] << 8);
-          };
-          auto field = [&](int i, int r) -> unsigned {         // table decode: the lane's 4 codes
-            const unsigned* w = reinterpret_cast<const unsigned*>(s_codes + i * kRunBytes + r * kRowBytes);
-            return __funnelshift_r(w[tb_word], w[tb_next], tb_shift);
-          };
-          // value = fl(scale * signed level), then the rounded add: the decode as defined
-          auto table_accumulate = [&](float sc, unsigned f0, unsigned f1) {
+        for (int c = 0; c < 2 * ROWS; ++c) a[c] = make_float2(0.0f, 0.0f);
+        auto window = [&](int i, int r) -> unsigned {       // 3-bit codes: the lane's 16-bit window
+          const unsigned char* q = s_codes + i * kRunBytes + r * kRowBytes;
+          return (unsigned)q[0] | ((unsigned)q[1] << 8);
+        };
+        auto field = [&](int i, int r) -> unsigned {         // table decode: the lane's 4 codes
+          const unsigned* w = reinterpret_cast<const unsigned*>(s_codes + i * kRunBytes + r * kRowBytes);
+          return __funnelshift_r(w[tb_word], w[tb_next], tb_shift);
+        };
+        // value = fl(scale * signed level), then the rounded add: the decode as defined
+        // (rows 2q and 2q + 1 go to accumulators a[4q] .. a[4q + 3]: two per row)
+        auto table_accumulate = [&](float sc, unsigned f0, unsigned f1, int q) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
-              const float v0 = __fmul_rn(sc, s_lut[(f0 >> (c * gb)) & tb_cmask]);
-              const float v1 = __fmul_rn(sc, s_lut[(f1 >> (c * gb)) & tb_cmask]);
-              float2& r0 = a[c >> 1];                          // row 0: a[0], a[1]; row 1: a[2], a[3]
-              float2& r1 = a[2 + (c >> 1)];
-              if (c & 1) { r0.y = __fadd_rn(r0.y, v0); r1.y = __fadd_rn(r1.y, v1); }
-              else       { r0.x = __fadd_rn(r0.x, v0); r1.x = __fadd_rn(r1.x, v1); }
-            }
-          };
-          auto contribute = [&](int i) {
+          for (int c = 0; c < 4; ++c) {
+            const float v0 = __fmul_rn(sc, s_lut[(f0 >> (c * gb)) & tb_cmask]);
+            const float v1 = __fmul_rn(sc, s_lut[(f1 >> (c * gb)) & tb_cmask]);
+            float2& r0 = a[4 * q + (c >> 1)];
+            float2& r1 = a[4 * q + 2 + (c >> 1)];
+            if (c & 1) { r0.y = __fadd_rn(r0.y, v0); r1.y = __fadd_rn(r1.y, v1); }
+            else       { r0.x = __fadd_rn(r0.x, v0); r1.x = __fadd_rn(r1.x, v1); }
+          }
+        };
+        auto row_pair = [&](int q) -> float2(&)[4] { return *reinterpret_cast<float2(*)[4]>(&a[4 * q]); };
+        auto contribute = [&](int i) {
+          const float2 sc = s_scale[i];
+#pragma unroll
+          for (int q = 0; q < ROWS / 2; ++q) {
             if constexpr (GB == 2) {
-              decode_accumulate(s_scale[i], s_codes[i * kRunBytes], s_codes[i * kRunBytes + kRowBytes], k01,
-                                k23, mg, a);
+              decode_accumulate(sc, s_codes[i * kRunBytes + 2 * q * kRowBytes],
+                                s_codes[i * kRunBytes + (2 * q + 1) * kRowBytes], k01, k23, mg, row_pair(q));
             } else if constexpr (GB == 3) {
-              decode_accumulate5<false>(s_scale[i], window(i, 0), window(i, 1), fl, a);
+              decode_accumulate5<false>(sc, window(i, 2 * q), window(i, 2 * q + 1), fl, row_pair(q));
             } else {
-              table_accumulate(s_scale[i].x, field(i, 0), field(i, 1));
+              table_accumulate(sc.x, field(i, 2 * q), field(i, 2 * q + 1), q);
             }
-          };
-          // ballot b: one bit per slot of workers b * v_per_ballot ... ; a slot beyond the
-          // window's pieces or the last worker votes "nothing"
-          const unsigned char* v_base = st + kCodesOff + v_off;
-          auto vote = [&](int b) -> unsigned {
-            const int i = b * v_per_ballot + v_worker0;
-            bool nz = false;
-            if (v_piece_ok && i < n) {
-              const uint4 w = *reinterpret_cast<const uint4*>(v_base + i * kRunBytes);
-              nz = (((w.x ^ kz[0]) | (w.y ^ kz[1])) | ((w.z ^ kz[2]) | (w.w ^ kz[3]))) != 0u;
-            }
-            return __ballot_sync(0xffffffffu, nz);
-          };
-          auto decode_live = [&](int b, unsigned bal) {        // the live workers of one ballot, in order
-            while (bal) {
-              const int g = (__ffs((int)bal) - 1) >> sl_log;
-              bal &= ~(v_gmask << (g << sl_log));
-              contribute(b * v_per_ballot + g);
-            }
-          };
-          if (tiny) {
-            // rare: every worker, products rounded before they are added
+          }
+        };
+        // ballot b: one bit per slot of workers b * v_per_ballot ... ; a slot beyond the
+        // window's pieces or the last worker votes "nothing"
+        const unsigned char* v_base = st + kCodesOff + v_off;
+        auto vote = [&](int b) -> unsigned {
+          const int i = b * v_per_ballot + v_worker0;
+          bool nz = false;
+          if (v_piece_ok && i < n) {
+            const uint4 w = *reinterpret_cast<const uint4*>(v_base + i * kRunBytes);
+            nz = (((w.x ^ kz[0]) | (w.y ^ kz[1])) | ((w.z ^ kz[2]) | (w.w ^ kz[3]))) != 0u;
+          }
+          return __ballot_sync(0xffffffffu, nz);
+        };
+        auto for_each_live = [&](int b, unsigned bal, auto&& fn) {   // live workers of one ballot, in order
+          while (bal) {
+            const int g = (__ffs((int)bal) - 1) >> sl_log;
+            bal &= ~(v_gmask << (g << sl_log));
+            fn(b * v_per_ballot + g);
+          }
+        };
+        if (tiny) {
+          // rare: every worker, products rounded before they are added
 #pragma unroll 1
-            for (int i = 0; i < n; ++i)
-              decode_accumulate5<true>(s_scale[i], window(i, 0), window(i, 1), fl, a);
-          } else if constexpr (NW > 0 && GB > 0) {
-            constexpr int kBallots = (NW * 2 * vote_pieces_pow2(GB) + 31) / 32;
-            unsigned bal[kBallots];
-            int live = 0;
+          for (int i = 0; i < n; ++i)
 #pragma unroll
-            for (int b = 0; b < kBallots; ++b) {
-              bal[b] = vote(b);
-              unsigned t = bal[b];                             // one bit per live worker
-              t |= t >> 1;
-              t |= t >> 2;
-              if (GB == 3) t |= t >> 4;
-              live += __popc(t & (GB == 2 ? 0x11111111u : 0x01010101u));
+            for (int q = 0; q < ROWS / 2; ++q)
+              decode_accumulate5<true>(s_scale[i], window(i, 2 * q), window(i, 2 * q + 1), fl, row_pair(q));
+        } else if constexpr (NW > 0 && GB > 0) {
+          constexpr int kSlots = ROWS * vote_pieces_pow2(GB);      // v_slots, at compile time
+          constexpr int kBallots = (NW * kSlots + 31) / 32;
+          unsigned bal[kBallots];
+          int live = 0;
+#pragma unroll
+          for (int b = 0; b < kBallots; ++b) {
+            bal[b] = vote(b);
+            unsigned t = bal[b];                             // folded to one bit per live worker
+            t |= t >> 1;
+            t |= t >> 2;
+            if (kSlots >= 8) t |= t >> 4;
+            if (kSlots >= 16) t |= t >> 8;
+            live += __popc(t & (kSlots == 4 ? 0x11111111u : kSlots == 8 ? 0x01010101u : 0x00010001u));
+          }
+          bool done = false;
+          if constexpr (GB == 2 && NW <= 32) {
+            // Between "a few live workers" and "codes everywhere": a live worker still has
+            // level 0 in nearly all of its bytes.  Each lane notes, per row, which live workers
+            // have anything in ITS byte; the warp then works in rounds, lane by lane taking its
+            // next such worker (increasing worker order per lane, which is all the sum's order
+            // asks for: different lanes hold different elements).  A lane with nothing left
+            // decodes a byte of level-0 codes, which adds +0.  The rounds are the largest
+            // number of such workers any lane has, usually a fraction of the live workers.
+            if (live >= 3 && dense_tiles_left <= 0) {
+              unsigned mk[ROWS];
+#pragma unroll
+              for (int r = 0; r < ROWS; ++r) mk[r] = 0u;
+#pragma unroll
+              for (int b = 0; b < kBallots; ++b)
+                for_each_live(b, bal[b], [&](int i) {
+#pragma unroll
+                  for (int r = 0; r < ROWS; ++r)
+                    mk[r] |= (s_codes[i * kRunBytes + r * kRowBytes] != 0x55u ? 1u : 0u) << i;
+                });
+              int rounds[ROWS], total_rounds = 0;
+#pragma unroll
+              for (int r = 0; r < ROWS; ++r) {
+                rounds[r] = (int)__reduce_max_sync(0xffffffffu, (unsigned)__popc(mk[r]));
+                total_rounds += rounds[r];
+              }
+              if (3 * total_rounds <= ROWS * live) {
+                auto round = [&](unsigned& m, int row_off, float2& lo, float2& hi) {
+                  const bool has = m != 0u;
+                  const int i = has ? __ffs((int)m) - 1 : 0;
+                  m &= m - 1u;
+                  const unsigned byte = has ? (unsigned)s_codes[i * kRunBytes + row_off] : 0x55u;
+                  const float2 sc = s_scale[i];
+                  lo = fma2_rn(code_pair_minus_bias<0x03u, 0x0cu>(byte, mg[0], mg[1], k01), sc, lo);
+                  hi = fma2_rn(code_pair_minus_bias<0x30u, 0xc0u>(byte, mg[2], mg[3], k23), sc, hi);
+                };
+#pragma unroll
+                for (int r = 0; r < ROWS; ++r)
+                  for (int k = 0; k < rounds[r]; ++k) round(mk[r], r * kRowBytes, a[2 * r], a[2 * r + 1]);
+                done = true;
+                dense_span = 8;
+              } else {
+                // codes too dense for rounds to pay: stop looking for a while (16, 32, ... 1024 tiles)
+                dense_span = dense_span < 1024 ? 2 * dense_span : 1024;
+                dense_tiles_left = dense_span;
+              }
             }
+            --dense_tiles_left;
+          }
+          if (!done) {
             if (4 * live >= 3 * NW) {
               // nearly every worker has something to add: the unrolled loop over all of them
 #pragma unroll kUnroll
               for (int i = 0; i < NW; ++i) contribute(i);
             } else {
 #pragma unroll
-              for (int b = 0; b < kBallots; ++b) decode_live(b, bal[b]);
+              for (int b = 0; b < kBallots; ++b) for_each_live(b, bal[b], contribute);
             }
-          } else {
-            // run-time worker count or code width: ballots taken and served one at a time
-            const int nb = (n * v_slots + 31) >> 5;
-            for (int b = 0; b < nb; ++b) decode_live(b, vote(b));
           }
-          // the tile's state into registers; pads beyond the tile's length are not used
-          const float* sx = reinterpret_cast<const float*>(st + kStageHeaderBytes) + gt * 4;
+        } else {
+          // run-time worker count or code width: ballots taken and served one at a time
+          const int nb = (n * v_slots + 31) >> 5;
+          for (int b = 0; b < nb; ++b) for_each_live(b, vote(b), contribute);
+        }
+        // the tile's state into registers; pads beyond the tile's length are not used
+        const float* sx = reinterpret_cast<const float*>(st + kStageHeaderBytes) + gt * 4;
 #pragma unroll
-          for (int r = 0; r < 2; ++r) {
-            if (r == 1 && !act1) break;
-            x4[r] = *reinterpret_cast<const float4*>(sx + r * (kPipeTile / 2));
-            if constexpr (SERVER_MOMENTS) {
-              m4[r] = *reinterpret_cast<const float4*>(sx + kPipeTile + r * (kPipeTile / 2));
-              v4[r] = *reinterpret_cast<const float4*>(sx + 2 * kPipeTile + r * (kPipeTile / 2));
-            }
+        for (int r = 0; r < ROWS; ++r) {
+          if (r > 0 && !active(r)) break;
+          x4[r] = *reinterpret_cast<const float4*>(sx + r * kPipeRowElems);
+          if constexpr (SERVER_MOMENTS) {
+            m4[r] = *reinterpret_cast<const float4*>(sx + kTile + r * kPipeRowElems);
+            v4[r] = *reinterpret_cast<const float4*>(sx + 2 * kTile + r * kPipeRowElems);
           }
         }
-        // everything this warp needs of the stage is in registers: hand it back
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&ps->empty[s]);
-        if (act0) {
-          float2 d[4];
-          if (inv_n_exact) {
-            const float2 inv = make_float2(p.inv_nf, p.inv_nf);
+      }
+      // everything this warp needs of the stage is in registers: hand it back
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&ps->empty[s]);
+      if (act0) {
+        float2 d[2 * ROWS];
+        if (inv_n_exact) {
+          const float2 inv = make_float2(p.inv_nf, p.inv_nf);
 #pragma unroll
-            for (int c = 0; c < 4; ++c) d[c] = mul2_rn(a[c], inv);
+          for (int c = 0; c < 2 * ROWS; ++c) d[c] = mul2_rn(a[c], inv);
+        } else {
+#pragma unroll
+          for (int c = 0; c < 2 * ROWS; ++c) d[c] = make_float2(__fdiv_rn(a[c].x, p.nf), __fdiv_rn(a[c].y, p.nf));
+        }
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r) {
+          if (r > 0 && !active(r)) break;
+          const long long e0 = hd.off + r * kPipeRowElems;
+          float xx[4];
+          if constexpr (SERVER_MOMENTS) {
+            float2 m01 = make_float2(m4[r].x, m4[r].y), m23 = make_float2(m4[r].z, m4[r].w);
+            float2 v01 = make_float2(v4[r].x, v4[r].y), v23 = make_float2(v4[r].z, v4[r].w);
+            moments2(p.h, d[2 * r], m01, v01);
+            moments2(p.h, d[2 * r + 1], m23, v23);
+            xx[0] = __fsub_rn(x4[r].x, adam_step(p.h, m01.x, v01.x, p.alpha));
+            xx[1] = __fsub_rn(x4[r].y, adam_step(p.h, m01.y, v01.y, p.alpha));
+            xx[2] = __fsub_rn(x4[r].z, adam_step(p.h, m23.x, v23.x, p.alpha));
+            xx[3] = __fsub_rn(x4[r].w, adam_step(p.h, m23.y, v23.y, p.alpha));
+            st_f4(gm + e0, make_float4(m01.x, m01.y, m23.x, m23.y));
+            st_f4(gv + e0, make_float4(v01.x, v01.y, v23.x, v23.y));
           } else {
-#pragma unroll
-            for (int c = 0; c < 4; ++c) d[c] = make_float2(__fdiv_rn(a[c].x, p.nf), __fdiv_rn(a[c].y, p.nf));
+            xx[0] = __fsub_rn(x4[r].x, d[2 * r].x);
+            xx[1] = __fsub_rn(x4[r].y, d[2 * r].y);
+            xx[2] = __fsub_rn(x4[r].z, d[2 * r + 1].x);
+            xx[3] = __fsub_rn(x4[r].w, d[2 * r + 1].y);
           }
-#pragma unroll
-          for (int r = 0; r < 2; ++r) {
-            if (r == 1 && !act1) break;
-            const long long e0 = hd.off + r * (kPipeTile / 2);
-            float xx[4];
-            if constexpr (SERVER_MOMENTS) {
-              float2 m01 = make_float2(m4[r].x, m4[r].y), m23 = make_float2(m4[r].z, m4[r].w);
-              float2 v01 = make_float2(v4[r].x, v4[r].y), v23 = make_float2(v4[r].z, v4[r].w);
-              moments2(p.h, d[2 * r], m01, v01);
-              moments2(p.h, d[2 * r + 1], m23, v23);
-              xx[0] = __fsub_rn(x4[r].x, adam_step(p.h, m01.x, v01.x, p.alpha));
-              xx[1] = __fsub_rn(x4[r].y, adam_step(p.h, m01.y, v01.y, p.alpha));
-              xx[2] = __fsub_rn(x4[r].z, adam_step(p.h, m23.x, v23.x, p.alpha));
-              xx[3] = __fsub_rn(x4[r].w, adam_step(p.h, m23.y, v23.y, p.alpha));
-              st_f4(p.m + e0 + gt * 4, make_float4(m01.x, m01.y, m23.x, m23.y));
-              st_f4(p.v + e0 + gt * 4, make_float4(v01.x, v01.y, v23.x, v23.y));
-            } else {
-              xx[0] = __fsub_rn(x4[r].x, d[2 * r].x);
-              xx[1] = __fsub_rn(x4[r].y, d[2 * r].y);
-              xx[2] = __fsub_rn(x4[r].z, d[2 * r + 1].x);
-              xx[3] = __fsub_rn(x4[r].w, d[2 * r + 1].y);
-            }
-            st_f4(p.x + e0 + gt * 4, make_float4(xx[0], xx[1], xx[2], xx[3]));
+          st_f4(gx + e0, make_float4(xx[0], xx[1], xx[2], xx[3]));
+          if constexpr (XB == 2) {
+            broadcast_row_ternary(xx, p.wcodes + ((e0 + gwarp * 128) >> 2),
+                                  p.wresid ? p.wresid + e0 + gt * 4 : nullptr, lane);
+          } else {
             if (p.kx >= 0)
               broadcast_row(xx, p.kx, p.xbits, p.wcodes, p.wresid, e0 + gt * 4, e0 + gwarp * 128, lane);
           }
         }
       }
-      if (++s == stages) { s = 0; ph ^= 1u; }
+      s += kPipeGroups;
+      if (s >= stages) { s -= stages; ph ^= 1u; }
     }
   }
   __syncthreads();

@@ -14,7 +14,7 @@
 // element this moves g, e in and e', the packed code out: 12 + b_g / 8 bytes (28 + b_g / 8
 // with m, v read and written), the least the method allows.
 //
-// The resident tiles of all workers are numbered worker-major, t = worker * TR + j
+// The resident tiles of the call's workers are numbered worker-major, t = worker * TR + j
 // (j: index in the per-vector list of resident tiles), so the tiles of a pair are
 // consecutive.  Tile t belongs to CTA t mod gridDim.x; a CTA takes its tiles in
 // increasing order and its i-th tile lives in slot i mod slots.  Per CTA, one per SM:
@@ -74,7 +74,7 @@ struct WorkerResidentParams {
   unsigned* done;         // [n][S] tiles counted per pair, zeroed before the launch (as are the scales)
   unsigned long long* words;  // [n][S][gridDim.x] or nullptr: per (pair, CTA) {tiles : 32, max |u| bits : 32},
                               // zeroed before the launch; when given, it replaces `done` and the atomics
-  long long total;        // n * TR resident tiles in all
+  long long total;        // resident tiles of the call: its workers x TR
   int TR;                 // resident tiles per worker
   int slots;              // slots of the CTA's ring (a pair gives a CTA fewer tiles than this)
   int estages;            // stages of the e ring
@@ -204,18 +204,21 @@ worker_resident_kernel(const WorkerResidentParams rp) {
              mbar_wait_bounded(&ps->e_empty[s], ph ^ 1u, abort_flag, p.status, spin);
         if (ok) {
           RLoadHeader* hd = &ps->load_hd[i & (kRHeaders - 1)];
-          hd->pair = (long long)worker * p.S + cur.seg;
+          // `worker` counts from the first worker of this call: g holds only the call's
+          // workers, every other array all n of them
+          hd->pair = (long long)(p.worker_begin + worker) * p.S + cur.seg;
           hd->slot = slot;
           hd->count = cur.count;
           hd->publish = publish;
           hd->max_bits = 0u;
           const unsigned bytes = (unsigned)cur.count * 4u;
-          const long long eo = (long long)worker * p.D + cur.off;
+          const long long eo = (long long)(p.worker_begin + worker) * p.D + cur.off;
           hd->elem = eo;
           hd->off = cur.off;
           unsigned char* st = ering_base + (size_t)s * kStageBytes;
           mbar_arrive_expect_tx(&ps->e_full[s], (WM ? 4u : 2u) * bytes);
-          bulk_load(slot_base + (size_t)slot * kRSlotBytes, p.g + eo, bytes, &ps->e_full[s]);
+          bulk_load(slot_base + (size_t)slot * kRSlotBytes, p.g + (long long)worker * p.D + cur.off, bytes,
+                    &ps->e_full[s]);
           bulk_load(st, p.e + eo, bytes, &ps->e_full[s]);
           if constexpr (WM) {
             bulk_load(st + kRSlotBytes, p.m + eo, bytes, &ps->e_full[s]);
@@ -291,7 +294,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
       int slot = 0;
       for (long long i = 0; i < my_tiles; ++i) {
         const RTile cur = rp.rtiles[j];
-        const long long pair = (long long)worker * p.S + cur.seg;
+        const long long pair = (long long)(p.worker_begin + worker) * p.S + cur.seg;
         if (pair != ready_pair) {                        // warp-uniform
           ok = false;
           if constexpr (WORDS) {
@@ -357,7 +360,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
             cd->off = cur.off;
             cd->slot = slot;
             cd->count = cur.count;
-            cd->worker = worker;
+            cd->worker = p.worker_begin + worker;
             cd->scale_bits = ready_scale;
             mbar_arrive(&ps->cmd_full[cs]);
           }
