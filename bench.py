@@ -74,6 +74,9 @@ def parse_args():
     ap.add_argument("--kg", type=int, default=None)
     ap.add_argument("--kx", type=int, default=None)
     ap.add_argument("--single-scale", action="store_true", help="one max-abs scale per worker")
+    ap.add_argument("--grad", default=None,
+                    help="gradient distribution in place of the workload's, e.g. gauss_clip:5 (Gaussian clipped "
+                         "at 5 sigma: about 1.2 %% of the ternary codes non-zero), gauss_clip:4 (4.6 %%), gauss_clip:2 (32 %%)")
     ap.add_argument("--scale-block-log2", type=int, default=0,
                     help="one max-abs scale per block of 2^K elements of a tensor (0: per tensor)")
     ap.add_argument("--weight-decay", type=float, default=0.0,
@@ -102,6 +105,8 @@ def get_workload(args):
         kw["kx"] = args.kx
     if args.single_scale:
         kw["per_tensor_scale"] = False
+    if args.grad:
+        kw["grad"] = args.grad
     if args.scale_block_log2 > 0:
         kw["scale_block"] = 1 << args.scale_block_log2
     return w.with_(**kw) if kw else w
@@ -289,6 +294,23 @@ def job_value(d: int, n_workers: int, world: int, ms_per_step: float) -> float:
 
 # ----------------------------------------------------------------------------- the CUDA path
 
+def alu_decode_peak():
+    """Codes per second the decode of the server pass could sustain if nothing but its two
+    busiest pipes mattered: a ternary code costs one logic operation (16 lanes per scheduler,
+    2 cycles per warp instruction) and half an add.f32x2 plus half an fma.f32x2 (2 cycles per
+    warp instruction each on the 32-lane fp32 pipe), so a scheduler retires 32 codes per 2
+    cycles on either pipe: 64 codes per clock and SM at the maximum SM clock."""
+    import torch
+    props = torch.cuda.get_device_properties(torch.cuda.current_device())
+    mhz = 1965.0
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as f:
+            mhz = float(json.load(f).get("sm_max_mhz", mhz))
+    except Exception:
+        pass
+    return props.multi_processor_count * 64.0 * mhz * 1e6
+
+
 def kernel_table(prof, w, placement_name, q, weight_decay, peak):
     """Per kernel: launches, time, algorithmic bytes, achieved rate and its fractions."""
     D = q.D
@@ -304,6 +326,12 @@ def kernel_table(prof, w, placement_name, q, weight_decay, peak):
         kernels[name] = {"launches": int(cnt), "ms_per_launch": per, "share": ms / total_ms,
                          "algorithmic_bytes": bytes_, "achieved_gbs": gbs,
                          "frac": gbs / peak, "frac_of_nominal": gbs / NOMINAL_HBM_GBS}
+        if name == "server" and w.kg == 0:
+            # second roofline of the server pass: with dense codes (always, when the moments are on
+            # the workers) it is bound by the arithmetic of the decode, not by HBM
+            codes = float(w.n) * D / (per * 1e-3)
+            kernels[name]["alu"] = {"bound": "alu", "achieved": codes, "peak": alu_decode_peak(),
+                                    "unit": "codes/s", "frac": codes / alu_decode_peak()}
     return kernels
 
 
@@ -414,7 +442,9 @@ def config_records(args, dev, world, peak):
                            else "fits in L2: not HBM evidence"),
                     "kernels": {k: {"ms_per_launch": v["ms_per_launch"], "launches": v["launches"],
                                     "achieved_gbs": v["achieved_gbs"], "frac": v["frac"],
-                                    "frac_of_nominal": v["frac_of_nominal"]} for k, v in m.kernels.items()}})
+                                    "frac_of_nominal": v["frac_of_nominal"],
+                                    **({"alu_frac": v["alu"]["frac"]} if "alu" in v else {})}
+                                for k, v in m.kernels.items()}})
         m.close()
         del m
         torch.cuda.empty_cache()

@@ -249,10 +249,13 @@ int qadam_shard_cuts(const qadam_config* cfg, int32_t shards, int64_t* cuts);
 
 /* One whole step from HOST memory, for callers whose gradients live on the host:
  * copies g_host ([n][D], host, ideally pinned) into g_stage (device, [n][D],
- * caller-owned), runs qadam_worker_compress for all workers and
- * qadam_server_step, then copies the result back to out_host (host): the packed
- * broadcast (wcode_bytes) when kx >= 0, else x (4*D bytes).  Waits for the
- * stream before returning.  out_host may be NULL to skip the read-back. */
+ * caller-owned) one worker at a time on a copy stream of the context's own (created by
+ * the first call), compressing worker i (qadam_worker_compress) while worker i + 1
+ * crosses the bus, then runs qadam_server_step and copies the result back to out_host
+ * (host): the packed broadcast (wcode_bytes) when kx >= 0, else x (4*D bytes).  Waits
+ * for the stream before returning.  out_host may be NULL to skip the read-back.  If a
+ * worker's call fails, the workers before it have been compressed: the context cannot
+ * continue with this step. */
 int qadam_step_host(qadam_ctx* ctx, int64_t step, const float* g_host, float* g_stage,
                     void* out_host, float lr_t);
 

@@ -220,6 +220,10 @@ struct qadam_ctx {
   RTile* d_rtiles = nullptr;
   Tile* d_btiles = nullptr;
   unsigned long long* d_words = nullptr;   // nullptr: one counter per pair instead
+  // qadam_step_host: the copy of worker i + 1 runs on a stream of its own while worker i is compressed
+  cudaStream_t copy_stream = nullptr;
+  cudaEvent_t copy_done[2] = {nullptr, nullptr};
+  cudaEvent_t stage_free = nullptr;
   // instrumentation: event pairs of the launches since the last read
   bool profiling = false;
   struct Timed { int kind; cudaEvent_t start, stop; };
@@ -876,11 +880,30 @@ int qadam_step_host(qadam_ctx* c, int64_t step, const float* g_host, float* g_st
   if (step != c->last_server_step + 1 || c->workers_done != 0 || c->range_open) return QADAM_ERR_STEP;
   const float alpha = lr_t < 0.0f ? c->cfg.lr : lr_t;
   if (!std::isfinite(alpha)) return QADAM_ERR_HYPER;
-  const size_t gbytes = sizeof(float) * (size_t)c->cfg.n * (size_t)c->geo.D;
-  if (!cuda_ok(cudaMemcpyAsync(g_stage, g_host, gbytes, cudaMemcpyHostToDevice, c->stream)))
+  // Worker by worker: the gradients of worker i + 1 cross the bus on a copy stream while the
+  // kernels of worker i run on the context's stream.
+  if (c->copy_stream == nullptr) {
+    if (!cuda_ok(cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking)) ||
+        !cuda_ok(cudaEventCreateWithFlags(&c->copy_done[0], cudaEventDisableTiming)) ||
+        !cuda_ok(cudaEventCreateWithFlags(&c->copy_done[1], cudaEventDisableTiming)) ||
+        !cuda_ok(cudaEventCreateWithFlags(&c->stage_free, cudaEventDisableTiming)))
+      return QADAM_ERR_CUDA;
+  }
+  // the staging buffer may still be read by work already on the context's stream
+  if (!cuda_ok(cudaEventRecord(c->stage_free, c->stream)) ||
+      !cuda_ok(cudaStreamWaitEvent(c->copy_stream, c->stage_free, 0)))
     return QADAM_ERR_CUDA;
-  int rc = qadam_worker_compress(c, step, g_stage, 0, c->cfg.n, lr_t);
-  if (rc != QADAM_OK) return rc;
+  const size_t wbytes = sizeof(float) * (size_t)c->geo.D;
+  int rc = QADAM_OK;
+  for (int i = 0; i < c->cfg.n; ++i) {
+    const size_t o = (size_t)i * (size_t)c->geo.D;
+    if (!cuda_ok(cudaMemcpyAsync(g_stage + o, g_host + o, wbytes, cudaMemcpyHostToDevice, c->copy_stream)) ||
+        !cuda_ok(cudaEventRecord(c->copy_done[i & 1], c->copy_stream)) ||
+        !cuda_ok(cudaStreamWaitEvent(c->stream, c->copy_done[i & 1], 0)))
+      return QADAM_ERR_CUDA;
+    rc = qadam_worker_compress(c, step, g_stage + o, i, 1, lr_t);
+    if (rc != QADAM_OK) return rc;
+  }
   rc = qadam_server_step(c, step, lr_t);
   if (rc != QADAM_OK) return rc;
   if (out_host) {
@@ -946,6 +969,9 @@ int qadam_destroy(qadam_ctx* c) {
     cudaEventDestroy(t.stop);
   }
   for (cudaEvent_t e : c->spare_events) cudaEventDestroy(e);
+  if (c->copy_stream) cudaStreamDestroy(c->copy_stream);
+  for (cudaEvent_t e : c->copy_done) if (e) cudaEventDestroy(e);
+  if (c->stage_free) cudaEventDestroy(c->stage_free);
   delete c;
   return QADAM_OK;
 }

@@ -22,7 +22,7 @@ class Workload:
     is_gamma: Tuple[bool, ...]        # normalisation scale vectors (init 1)
     n: int                            # simulated workers
     steps: int                        # optimizer steps T
-    grad: str                         # "gauss_worker" | "gauss_tensor" | "student_t_tensor" | "mixture"
+    grad: str                         # "gauss_worker" | "gauss_tensor" | "student_t_tensor" | "mixture" | "gauss_clip:<C>"
     w0: str                           # "gauss:<sigma>" | "he"
     kg: int = 0                       # gradient quantizer level parameter (-1: identity)
     kx: int = -1                      # weight quantizer level parameter (-1: none)

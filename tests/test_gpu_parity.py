@@ -513,3 +513,32 @@ def test_stochastic_operator_is_ternary_only():
     assert ei.value.code == -3
     with pytest.raises(qb.QAdamError):
         qb.QAdam([1000], 2, kg=-1, grid_g=qb.GRID_STOCHASTIC)
+
+
+# ---------------------------------------------------------------- the step from host buffers
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+@pytest.mark.parametrize("kx", [0, -1])
+def test_step_from_host_buffers(kx, placement):
+    """qadam_step_host (pinned host gradients in, worker by worker on a copy stream; packed
+    broadcast or x out) gives the bits of the two-call step and of the oracle."""
+    rng = np.random.default_rng(60 + kx + placement)
+    seg, n = [3 * 4096 + 640, 130, 70000, 1], 5
+    d = sum(seg)
+    x1 = (rng.standard_normal(d) * 0.2).astype(np.float32)
+    p = Pair(seg, n, 0, kx, placement, x1=x1)
+    D = p.gpu.D
+    g_stage = torch.zeros(n, D, device="cuda")
+    out_bytes = p.gpu.wcode_bytes if kx >= 0 else 4 * D
+    out_host = torch.zeros(out_bytes, dtype=torch.uint8).pin_memory()
+    for t in range(1, 4):
+        gp = p.cpu.to_padded(_rand_grads(rng, n, d))
+        g_host = torch.from_numpy(gp).pin_memory()
+        p.gpu.step_host(t, g_host.view(-1), g_stage, out_host)
+        p.cpu.step(gp, p.lr)
+        p.step_no = t
+        p.compare_worker_outputs()
+        p.compare_state()
+        want = p.cpu.wcodes if kx >= 0 else p.cpu.x.view(np.uint8)
+        assert np.array_equal(out_host.numpy()[:want.size], want)
+    p.close()
