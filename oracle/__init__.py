@@ -91,9 +91,9 @@ def lib():
         L.qo_quantize_grad_segment_stochastic.argtypes = [f32p, C.c_int64, C.c_int64, C.c_uint64, C.c_uint32,
                                                           C.c_uint32, f32p, i32p, f32p]
         L.qo_broadcast_weights.restype = C.c_int32
-        L.qo_broadcast_weights.argtypes = [pp, f32p, u8p, f32p]
+        L.qo_broadcast_weights.argtypes = [pp, f32p, u8p, f32p, f32p]
         L.qo_server_step.restype = C.c_int32
-        L.qo_server_step.argtypes = [pp, f32p, u8p, f32p, f32p, f32p, C.c_float, u8p, f32p]
+        L.qo_server_step.argtypes = [pp, f32p, u8p, f32p, f32p, f32p, C.c_float, u8p, f32p, f32p]
         L.qo_decode_weights.restype = C.c_int32
         L.qo_decode_weights.argtypes = [pp, u8p, f32p]
         _lib = L
@@ -205,7 +205,7 @@ class OracleState:
 
     def __init__(self, seg_len: Sequence[int], n: int, kg: int, kx: int, placement: int,
                  beta1: float, beta2: float, eps: float, grid_g: int = GRID_POW2,
-                 want_wresid: bool = False, seed: int = 0):
+                 want_wresid: bool = False, seed: int = 0, want_wfeedback: bool = False):
         self.seg_len = np.ascontiguousarray(seg_len, dtype=np.int64)
         self.seg_off, self.D = layout(self.seg_len)
         self.d = int(self.seg_len.sum())
@@ -227,6 +227,8 @@ class OracleState:
         self.gcodes = np.zeros((self.n, self.gcode_bytes), np.uint8)
         self.wcodes = np.zeros(self.wcode_bytes, np.uint8)
         self.wresid = np.zeros(D, np.float32) if want_wresid else None
+        # optional error buffer of the broadcast (sigma-delta form, beyond the paper): starts at zero
+        self.wfeedback = np.zeros(D, np.float32) if want_wfeedback else None
 
     # layout helpers -------------------------------------------------------
     def to_padded(self, logical: np.ndarray) -> np.ndarray:
@@ -255,7 +257,7 @@ class OracleState:
     def broadcast(self) -> None:
         lib().qo_broadcast_weights(C.byref(self._prob), _p(self.x, C.c_float),
                                    _p(self.wcodes, C.c_uint8) if self.kx >= 0 else None,
-                                   _p(self.wresid, C.c_float))
+                                   _p(self.wresid, C.c_float), _p(self.wfeedback, C.c_float))
 
     # step-dependent parameters -------------------------------------------------
     def set_moment_rates(self, beta_t: float, theta_t: float) -> None:
@@ -307,7 +309,7 @@ class OracleState:
             _p(self.m, C.c_float) if sm else None,
             _p(self.v, C.c_float) if sm else None, lr,
             _p(self.wcodes, C.c_uint8) if self.kx >= 0 else None,
-            _p(self.wresid, C.c_float))
+            _p(self.wresid, C.c_float), _p(self.wfeedback, C.c_float))
         if rc != 0:
             raise RuntimeError(f"qo_server_step failed: {rc}")
         self.step_no += 1

@@ -460,18 +460,37 @@ int32_t qo_worker_step(const qo_problem* p, const float* g, const float* xhat, f
 // READING (weight error feedback): the server keeps the full-precision x_t and
 // only the broadcast is quantized, so the part Q_x drops is never lost; the
 // residual is a derived quantity, written out only when asked for.
+// BEYOND THE PAPER (wfeedback, optional): a separate error buffer for the broadcast in
+// the manner of Algorithm 1's e for the gradients ("sigma-delta" form): what is sent is
+// Q_x(y) with y = x + e^w, and e^w <- y - Q_x(y), so that the quantization error of one
+// broadcast is carried into the next instead of being forgotten: the broadcasts then add
+// up to the master weights, sum_t Q_x(y_t) + e^w_{T+1} = sum_t x_t + e^w_1.  The master
+// copy x is not touched by it.  With a buffer, wresid (if asked for) is the new e^w.
 // ---------------------------------------------------------------------------
-int32_t qo_broadcast_weights(const qo_problem* p, const float* x, uint8_t* wcodes, float* wresid) {
+int32_t qo_broadcast_weights(const qo_problem* p, const float* x, uint8_t* wcodes, float* wresid,
+                             float* wfeedback) {
   if (p->kx < 0) return 0;
   const int bits = qo_weight_code_bits(p->kx);
   const int L = 1 << p->kx;
   std::vector<int32_t> q;
   std::vector<uint32_t> code;
+  std::vector<float> y, r;
   for (int32_t s = 0; s < p->S; ++s) {
     const int64_t off = p->seg_off[s], len = p->seg_len[s];
     const int64_t plen = round_up(len, kAlign);
     q.assign((size_t)len, 0);
-    quantize_weights(x + off, len, p->kx, q.data(), nullptr, wresid ? wresid + off : nullptr);
+    if (wfeedback) {
+      y.resize((size_t)len);
+      r.resize((size_t)len);
+      for (int64_t j = 0; j < len; ++j) y[j] = x[off + j] + wfeedback[off + j];
+      quantize_weights(y.data(), len, p->kx, q.data(), nullptr, r.data());
+      for (int64_t j = 0; j < len; ++j) {
+        wfeedback[off + j] = r[j];
+        if (wresid) wresid[off + j] = r[j];
+      }
+    } else {
+      quantize_weights(x + off, len, p->kx, q.data(), nullptr, wresid ? wresid + off : nullptr);
+    }
     code.assign((size_t)plen, (uint32_t)L);
     for (int64_t j = 0; j < len; ++j) code[j] = (uint32_t)(q[j] + L);
     if (wcodes) pack_bits(code.data(), plen, bits, wcodes + off * bits / 8);
@@ -490,7 +509,7 @@ int32_t qo_broadcast_weights(const qo_problem* p, const float* x, uint8_t* wcode
 // ---------------------------------------------------------------------------
 int32_t qo_server_step(const qo_problem* p, const float* scales, const uint8_t* codes,
                        float* x, float* m, float* v, float alpha,
-                       uint8_t* wcodes, float* wresid) {
+                       uint8_t* wcodes, float* wresid, float* wfeedback) {
   const Hyper h = make_hyper(p->beta, p->theta, p->eps);
   GradLevels G;
   if (p->kg >= 0 && !make_grad_levels(p->kg, p->grid_g, &G)) return -1;
@@ -531,7 +550,7 @@ int32_t qo_server_step(const qo_problem* p, const float* scales, const uint8_t* 
       }
     }
   }
-  return qo_broadcast_weights(p, x, wcodes, wresid);
+  return qo_broadcast_weights(p, x, wcodes, wresid, wfeedback);
 }
 
 // Decode a packed weight broadcast back to values (what a worker receives).

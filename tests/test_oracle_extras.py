@@ -163,3 +163,50 @@ def test_step_dependent_rates_follow_a_textbook_loop(oracle):
     st2.step(st2.to_padded(g[0])[None, :], 1e-3)
     assert np.array_equal(st2.to_logical(st2.v[0]), f(0.5) * (g[0] * g[0]))
     assert np.array_equal(st2.to_logical(st2.m[0]), g[0])
+
+
+# ---------------------------------------------------------------- error feedback for the broadcast
+
+@pytest.mark.parametrize("kx", [0, 2, 6])
+def test_weight_feedback_buffer_carries_the_broadcast_error(oracle, kx):
+    """The optional error buffer of the broadcast (beyond the paper): what is sent is Q_x(x + e^w)
+    and e^w <- (x + e^w) - Q_x(x + e^w).  Pins: each step follows that definition with Q_x from
+    the rational brute force; the broadcasts telescope, sum_t Q_x(y_t) + e^w_{T+1} = sum_t x_t;
+    e^w stays within half a grid step; the master weights are exactly those of a run without
+    the buffer; and without the buffer nothing changes.  (Weights stay inside [-1/2, 1/2].)"""
+    from _util import brute_qx
+    rng = np.random.default_rng(70 + kx)
+    seg, n, T = [200, 70, 130], 2, 6
+    d = sum(seg)
+    x1 = np.clip(rng.standard_normal(d) * 0.15, -0.4, 0.4).astype(np.float32)
+    a = oracle.OracleState(seg, n, 0, kx, 0, 0.9, 0.999, 1e-8, want_wfeedback=True, want_wresid=True)
+    b = oracle.OracleState(seg, n, 0, kx, 0, 0.9, 0.999, 1e-8)
+    a.set_weights(x1)
+    b.set_weights(x1)
+    step = np.float32(2.0 ** -(kx + 1))
+    sent_sum = np.zeros(a.D, np.float64)
+    x_sum = np.zeros(a.D, np.float64)
+    ew_before = np.zeros(a.D, np.float32)
+    for t in range(T + 1):
+        # the broadcast that has just been emitted is Q_x(x + e^w before it)
+        y = a.x + ew_before
+        q = np.zeros(a.D, np.int32)
+        for off, ln in zip(a.seg_off.tolist(), a.seg_len.tolist()):
+            q[off:off + ln] = brute_qx(y[off:off + ln], kx)
+        xhat = q.astype(np.float32) * step
+        assert np.array_equal(a.decoded_weights(), xhat)
+        assert np.array_equal(a.wfeedback, y - xhat) and np.array_equal(a.wresid, a.wfeedback)
+        inside = np.abs(y) <= 0.5                  # beyond the grid's end Q_x clips and the error is larger
+        assert np.max(np.abs(a.wfeedback[inside])) <= 2.0 ** -(kx + 2) + 1e-12
+        sent_sum += xhat
+        x_sum += a.x
+        assert np.array_equal(a.x, b.x), "the master copy does not depend on the buffer"
+        ew_before = a.wfeedback.copy()
+        if t < T:
+            g = a.to_padded((rng.standard_normal((n, d)) * 0.01).astype(np.float32))
+            a.step(g, 1e-2)
+            b.step(g, 1e-2)
+    assert np.max(np.abs(sent_sum + a.wfeedback - x_sum)) < 1e-5
+    # without the buffer the broadcast is Q_x(x), and it drifts from the running mean of x further
+    plain_err = np.abs(b.decoded_weights() - b.x).max()
+    assert plain_err <= 2.0 ** -(kx + 2)
