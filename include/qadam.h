@@ -166,6 +166,13 @@ typedef struct {
                                  the library keeps tables here between calls: do not touch it   */
   size_t workspace_bytes;
   uint32_t* status;           /* one word; qadam_create clears it                                 */
+  float* wfeedback;           /* [D] optional (NULL: off; needs kx >= 0), zeros at creation.  An
+                                 error buffer for the broadcast, which the paper does not have
+                                 (its server keeps the master copy and forgets what Q_x drops):
+                                 what is broadcast becomes Q_x(y), y = x + wfeedback, and
+                                 wfeedback <- y - Q_x(y), so that successive broadcasts add up
+                                 to the master weights.  x itself is unaffected.  With it,
+                                 wresid (if given) receives the new wfeedback                    */
 } qadam_buffers;
 
 /* Sizes for a configuration.  Any output pointer may be NULL.

@@ -69,7 +69,7 @@ class QAdamBuffers(C.Structure):
         ("x", C.c_void_p), ("m", C.c_void_p), ("v", C.c_void_p), ("e", C.c_void_p),
         ("scales", C.c_void_p), ("gcodes", C.c_void_p), ("wcodes", C.c_void_p),
         ("wresid", C.c_void_p), ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
-        ("status", C.c_void_p),
+        ("status", C.c_void_p), ("wfeedback", C.c_void_p),
     ]
 
 
@@ -280,7 +280,7 @@ class QAdam:
                  eps: float = 1e-8, lr: float = 1e-3, grid_g: int = GRID_POW2,
                  x1: Optional[torch.Tensor] = None, want_wresid: bool = False,
                  device: Optional[torch.device] = None, stream: Optional[torch.cuda.Stream] = None,
-                 seed: int = 0, options: Optional[QAdamOptions] = None):
+                 seed: int = 0, options: Optional[QAdamOptions] = None, want_wfeedback: bool = False):
         load_library()
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2004_14180_b200 needs a CUDA device; there is no CPU path")
@@ -309,6 +309,7 @@ class QAdam:
             self.gcodes = z(self.n, self.gcode_bytes, dtype=torch.uint8)
             self.wcodes = z(max(self.wcode_bytes, 16), dtype=torch.uint8)
             self.wresid = z(D) if want_wresid else None
+            self.wfeedback = z(D) if want_wfeedback else None      # error buffer of the broadcast (optional)
             self.workspace = z(sz["workspace_bytes"] + 256, dtype=torch.uint8)
             self.status = z(4, dtype=torch.int32)
             if x1 is not None:
@@ -320,7 +321,8 @@ class QAdam:
                 wcodes=self.wcodes.data_ptr() if kx >= 0 else None,
                 wresid=self.wresid.data_ptr() if want_wresid else None,
                 workspace=ws_ptr, workspace_bytes=sz["workspace_bytes"],
-                status=self.status.data_ptr())
+                status=self.status.data_ptr(),
+                wfeedback=self.wfeedback.data_ptr() if want_wfeedback else None)
             # buffers were filled on torch's current stream; the context may use another
             torch.cuda.current_stream(self.device).synchronize()
             self.ctx = (qadam_create(self.cfg, self.bufs) if options is None

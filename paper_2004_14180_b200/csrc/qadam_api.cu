@@ -400,6 +400,7 @@ ServerParams make_server_params(const qadam_ctx* c, float alpha) {
   p.gcodes = static_cast<const unsigned char*>(c->buf.gcodes);
   p.wcodes = static_cast<unsigned char*>(c->buf.wcodes);
   p.wresid = c->buf.wresid;
+  p.wfeedback = c->buf.wfeedback;
   p.tiles = c->d_tiles;
   p.D = c->geo.D;
   p.gcode_bytes = (long long)c->geo.gcode_bytes;
@@ -471,7 +472,8 @@ int qadam_create_ex(const qadam_config* cfg, const qadam_buffers* b, const qadam
       !b->status || (quant_x && !b->wcodes)) {
     delete c; return QADAM_ERR_NULL;
   }
-  const void* ptrs[] = {b->x, b->m, b->v, b->e, b->scales, b->gcodes, b->wcodes, b->wresid, b->status};
+  if (b->wfeedback && !quant_x) { delete c; return QADAM_ERR_LEVEL; }     // a feedback buffer needs a weight quantizer
+  const void* ptrs[] = {b->x, b->m, b->v, b->e, b->scales, b->gcodes, b->wcodes, b->wresid, b->wfeedback, b->status};
   for (const void* p : ptrs) {
     if (p && !aligned(p, p == b->status || p == b->scales ? 4 : 16)) { delete c; return QADAM_ERR_ALIGN; }
   }

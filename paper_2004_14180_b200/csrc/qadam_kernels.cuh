@@ -162,6 +162,7 @@ struct ServerParams {
   const unsigned char* gcodes;  // [n][gcode_bytes]
   unsigned char* wcodes; // [wcode_bytes] or nullptr
   float* wresid;         // [D] or nullptr
+  float* wfeedback;      // [D] or nullptr: error buffer of the broadcast (Q_x is applied to x + wfeedback)
   const Tile* tiles;
   long long D;
   long long gcode_bytes;
@@ -433,16 +434,26 @@ worker_identity_kernel(const WorkerParams p) {
 // ---------------------------------------------------------------------------
 // Q_x of 4 consecutive weights of one lane, packed row store, optional residual.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ void broadcast_row(const float xx[4], int kx, int xbits,
-                                              unsigned char* wcodes, float* wresid,
+// With an error buffer for the broadcast (wfeedback, not in the paper) the quantized value is
+// y = x + wfeedback and the buffer becomes y - Q_x(y).
+__device__ __forceinline__ void broadcast_row(const float xin[4], int kx, int xbits,
+                                              unsigned char* wcodes, float* wresid, float* wfeedback,
                                               long long elem, long long row_elem, int lane) {
   unsigned code[4];
+  float xx[4] = {xin[0], xin[1], xin[2], xin[3]};
   float xq[4];
+  if (wfeedback) {
+    const float4 ew = ld_f4(wfeedback + elem);
+    xx[0] = __fadd_rn(xx[0], ew.x); xx[1] = __fadd_rn(xx[1], ew.y);
+    xx[2] = __fadd_rn(xx[2], ew.z); xx[3] = __fadd_rn(xx[3], ew.w);
+  }
 #pragma unroll
   for (int c = 0; c < 4; ++c) code[c] = quantize_weight(xx[c], kx, xq[c]);
-  if (wresid) {
-    st_f4(wresid + elem, make_float4(__fsub_rn(xx[0], xq[0]), __fsub_rn(xx[1], xq[1]),
-                                     __fsub_rn(xx[2], xq[2]), __fsub_rn(xx[3], xq[3])));
+  if (wresid || wfeedback) {
+    const float4 r = make_float4(__fsub_rn(xx[0], xq[0]), __fsub_rn(xx[1], xq[1]),
+                                 __fsub_rn(xx[2], xq[2]), __fsub_rn(xx[3], xq[3]));
+    if (wresid) st_f4(wresid + elem, r);
+    if (wfeedback) st_f4(wfeedback + elem, r);
   }
   void* dst = wcodes + row_elem * xbits / 8;
   switch (xbits) {
@@ -466,7 +477,7 @@ weight_broadcast_kernel(const ServerParams p) {
       if (idx >= tile.count) continue;
       const float4 x4 = ld_f4(p.x + tile.off + idx);
       const float xx[4] = {x4.x, x4.y, x4.z, x4.w};
-      broadcast_row(xx, p.kx, p.xbits, p.wcodes, p.wresid, tile.off + idx,
+      broadcast_row(xx, p.kx, p.xbits, p.wcodes, p.wresid, p.wfeedback, tile.off + idx,
                     tile.off + r * kRowElems + warp * 128, lane);
     }
   }
@@ -621,7 +632,7 @@ server_step_kernel(const ServerParams p) {
       }
       st_f4(p.x + tile.off + idx, make_float4(xx[0], xx[1], xx[2], xx[3]));
       if (p.kx >= 0) {
-        broadcast_row(xx, p.kx, p.xbits, p.wcodes, p.wresid, tile.off + idx,
+        broadcast_row(xx, p.kx, p.xbits, p.wcodes, p.wresid, p.wfeedback, tile.off + idx,
                       tile.off + r * kRowElems + warp * 128, lane);
       }
     }

@@ -333,10 +333,17 @@ __host__ __device__ constexpr int vote_pieces_pow2(int gb) { return gb <= 2 ? 2 
 // packed store of the warp's row of 128 two-bit codes (32 bytes): the four codes of a lane
 // are one byte; two shuffle steps gather four lanes' bytes into a word, which lanes
 // 0, 4, ..., 28 store.  row_dst: address of the row's first code.
-__device__ __forceinline__ void broadcast_row_ternary(const float xx[4], unsigned char* row_dst,
-                                                      float* wresid_elem, int lane) {
+// wfeedback_elem (optional): the thread's 4 values of the broadcast's error buffer, see broadcast_row.
+__device__ __forceinline__ void broadcast_row_ternary(const float xin[4], unsigned char* row_dst,
+                                                      float* wresid_elem, float* wfeedback_elem, int lane) {
   unsigned field = 0;
+  float xx[4] = {xin[0], xin[1], xin[2], xin[3]};
   float xq[4];
+  if (wfeedback_elem) {
+    const float4 ew = ld_f4(wfeedback_elem);
+    xx[0] = __fadd_rn(xx[0], ew.x); xx[1] = __fadd_rn(xx[1], ew.y);
+    xx[2] = __fadd_rn(xx[2], ew.z); xx[3] = __fadd_rn(xx[3], ew.w);
+  }
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
     // midpoint 1/4, ties toward zero; code = level index + 1
@@ -344,9 +351,11 @@ __device__ __forceinline__ void broadcast_row_ternary(const float xx[4], unsigne
     xq[c] = up ? 0.5f : (down ? -0.5f : 0.0f);
     field |= (up ? 2u : (down ? 0u : 1u)) << (2 * c);
   }
-  if (wresid_elem) {
-    st_f4(wresid_elem, make_float4(__fsub_rn(xx[0], xq[0]), __fsub_rn(xx[1], xq[1]),
-                                   __fsub_rn(xx[2], xq[2]), __fsub_rn(xx[3], xq[3])));
+  if (wresid_elem || wfeedback_elem) {
+    const float4 r = make_float4(__fsub_rn(xx[0], xq[0]), __fsub_rn(xx[1], xq[1]),
+                                 __fsub_rn(xx[2], xq[2]), __fsub_rn(xx[3], xq[3]));
+    if (wresid_elem) st_f4(wresid_elem, r);
+    if (wfeedback_elem) st_f4(wfeedback_elem, r);
   }
   unsigned w = field | (__shfl_down_sync(0xffffffffu, field, 1) << 8);
   w |= __shfl_down_sync(0xffffffffu, w, 2) << 16;
@@ -757,10 +766,11 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
           st_f4(gx + e0, make_float4(xx[0], xx[1], xx[2], xx[3]));
           if constexpr (XB == 2) {
             broadcast_row_ternary(xx, p.wcodes + ((e0 + gwarp * 128) >> 2),
-                                  p.wresid ? p.wresid + e0 + gt * 4 : nullptr, lane);
+                                  p.wresid ? p.wresid + e0 + gt * 4 : nullptr,
+                                  p.wfeedback ? p.wfeedback + e0 + gt * 4 : nullptr, lane);
           } else {
             if (p.kx >= 0)
-              broadcast_row(xx, p.kx, p.xbits, p.wcodes, p.wresid, e0 + gt * 4, e0 + gwarp * 128, lane);
+              broadcast_row(xx, p.kx, p.xbits, p.wcodes, p.wresid, p.wfeedback, e0 + gt * 4, e0 + gwarp * 128, lane);
           }
         }
       }

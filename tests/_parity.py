@@ -30,14 +30,15 @@ class Pair:
     """One problem held twice: `gpu` (qb.QAdam) and `cpu` (oracle.OracleState)."""
 
     def __init__(self, seg_len, n, kg, kx, placement, x1=None, grid_g=0, beta1=0.9, beta2=0.999,
-                 eps=1e-8, lr=1e-3, want_wresid=False, options=None, seed=0):
+                 eps=1e-8, lr=1e-3, want_wresid=False, options=None, seed=0, want_wfeedback=False):
         self.lr = lr
         x1_t = None if x1 is None else torch.as_tensor(x1, dtype=torch.float32)
         self.gpu = qb.QAdam(seg_len, n, kg=kg, kx=kx, placement=placement, beta1=beta1, beta2=beta2,
                             eps=eps, lr=lr, grid_g=grid_g, x1=x1_t, want_wresid=want_wresid,
-                            options=options, seed=seed)
+                            options=options, seed=seed, want_wfeedback=want_wfeedback)
         self.cpu = oracle.OracleState(seg_len, n, kg, kx, placement, beta1, beta2, eps,
-                                      grid_g=grid_g, want_wresid=want_wresid, seed=seed)
+                                      grid_g=grid_g, want_wresid=want_wresid, seed=seed,
+                                      want_wfeedback=want_wfeedback)
         if x1 is not None:
             self.cpu.set_weights(np.asarray(x1, dtype=np.float32))
         else:
@@ -97,6 +98,8 @@ class Pair:
             assert np.array_equal(g.wcodes.cpu().numpy()[:c.wcode_bytes], c.wcodes), "wcodes differ"
         if c.wresid is not None:
             assert bits_equal(g.wresid.cpu().numpy(), c.wresid), "wresid differs"
+        if c.wfeedback is not None:
+            assert bits_equal(g.wfeedback.cpu().numpy(), c.wfeedback), "wfeedback differs"
 
     def close(self):
         self.gpu.close()

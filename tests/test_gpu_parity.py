@@ -542,3 +542,40 @@ def test_step_from_host_buffers(kx, placement):
         want = p.cpu.wcodes if kx >= 0 else p.cpu.x.view(np.uint8)
         assert np.array_equal(out_host.numpy()[:want.size], want)
     p.close()
+
+
+# ---------------------------------------------------------------- error buffer for the broadcast
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+@pytest.mark.parametrize("kx,n,kg", [(0, 4, 0), (3, 5, 0), (6, 16, 1), (0, 70, 0), (2, 3, 3)])
+def test_weight_feedback_buffer(kx, n, kg, placement):
+    """The optional error buffer of the broadcast (Q_x applied to x + e^w, e^w <- what Q_x
+    dropped; not in the paper): through the pipelined pass with its ternary-weight path, the
+    generic path, the table decode and the plain kernel, one step served by ranges."""
+    import paper_2004_14180_b200 as qb
+    rng = np.random.default_rng(1200 + 10 * kx + n)
+    seg = [3 * 4096 + 640, 130, 9000, 1]
+    d = sum(seg)
+    x1 = (rng.standard_normal(d) * 0.2).astype(np.float32)
+    p = Pair(seg, n, kg, kx, placement, x1=x1, want_wfeedback=True, want_wresid=(kx == 3))
+    p.compare_state()                                   # the first broadcast already feeds the buffer
+    for t in range(1, 5):
+        g = _rand_grads(rng, n, d)
+        if t == 3:                                      # one step range by range
+            gp = p.cpu.to_padded(g)
+            p.gpu.worker_compress(t, torch.from_numpy(gp).cuda())
+            p.cpu.workers_step(gp, p.lr)
+            cuts = p.gpu.shard_cuts(3)
+            for r in (2, 0, 1):
+                p.gpu.server_step_range(t, cuts[r], cuts[r + 1])
+            p.gpu.finish_step(t)
+            p.cpu.server_step(p.lr)
+            p.step_no = t
+        else:
+            p.step(g)
+        p.compare_state()
+    assert float(p.gpu.wfeedback.abs().max()) > 0
+    p.close()
+    with pytest.raises(qb.QAdamError) as ei:
+        qb.QAdam([1000], 2, kg=0, kx=-1, want_wfeedback=True)      # nothing to feed back without Q_x
+    assert ei.value.code == -3
