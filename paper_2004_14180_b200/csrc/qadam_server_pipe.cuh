@@ -336,7 +336,6 @@ __host__ __device__ constexpr int vote_pieces_pow2(int gb) { return gb <= 2 ? 2 
 // wfeedback_elem (optional): the thread's 4 values of the broadcast's error buffer, see broadcast_row.
 __device__ __forceinline__ void broadcast_row_ternary(const float xin[4], unsigned char* row_dst,
                                                       float* wresid_elem, float* wfeedback_elem, int lane) {
-  unsigned field = 0;
   float xx[4] = {xin[0], xin[1], xin[2], xin[3]};
   float xq[4];
   if (wfeedback_elem) {
@@ -344,13 +343,24 @@ __device__ __forceinline__ void broadcast_row_ternary(const float xin[4], unsign
     xx[0] = __fadd_rn(xx[0], ew.x); xx[1] = __fadd_rn(xx[1], ew.y);
     xx[2] = __fadd_rn(xx[2], ew.z); xx[3] = __fadd_rn(xx[3], ew.w);
   }
+  // Level index q = [x > 1/4] - [x < -1/4] (midpoint 1/4, ties toward zero), code = q + 1,
+  // taken on the fp32 pipe, which has slots to spare when the integer pipe is busy decoding:
+  // sat(x 2^30 - 2^28) is 1 for every float above 1/4 (the smallest such difference times
+  // 2^30 is 32) and 0 for 1/4 and below, exactly; likewise for -1/4.  The four codes are
+  // gathered by exact multiply-adds (c0 + 4 c1 + 16 c2 + 64 c3 <= 170) and read out of the
+  // mantissa of 2^23 + that.
+  float cf[4];
 #pragma unroll
   for (int c = 0; c < 4; ++c) {
-    // midpoint 1/4, ties toward zero; code = level index + 1
-    const bool up = xx[c] > 0.25f, down = xx[c] < -0.25f;
-    xq[c] = up ? 0.5f : (down ? -0.5f : 0.0f);
-    field |= (up ? 2u : (down ? 0u : 1u)) << (2 * c);
+    float up, down;
+    asm("fma.rn.sat.f32 %0, %1, 0f4E800000, 0fCD800000;" : "=f"(up) : "f"(xx[c]));     // x * 2^30 - 2^28
+    asm("fma.rn.sat.f32 %0, %1, 0fCE800000, 0fCD800000;" : "=f"(down) : "f"(xx[c]));   // -x * 2^30 - 2^28
+    const float q = __fsub_rn(up, down);
+    xq[c] = __fmul_rn(0.5f, q);
+    cf[c] = __fadd_rn(q, 1.0f);
   }
+  const float packed = __fmaf_rn(__fmaf_rn(__fmaf_rn(cf[3], 4.0f, cf[2]), 4.0f, cf[1]), 4.0f, cf[0]);
+  const unsigned field = __float_as_uint(__fadd_rn(packed, 8388608.0f)) & 0xffu;
   if (wresid_elem || wfeedback_elem) {
     const float4 r = make_float4(__fsub_rn(xx[0], xq[0]), __fsub_rn(xx[1], xq[1]),
                                  __fsub_rn(xx[2], xq[2]), __fsub_rn(xx[3], xq[3]));
@@ -554,6 +564,8 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
     float* const gv = SERVER_MOMENTS ? p.v + gt * 4 : nullptr;
     int dense_tiles_left = 0;         // warp-uniform: tiles for which the search for sparse structure is skipped
     int dense_span = 8;
+    int all_live_left = 0;            // warp-uniform: tiles for which even the vote is skipped (every worker decoded)
+    int all_live_span = 4;
 
     int s = group;
     unsigned ph = 0;
@@ -642,18 +654,34 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
           constexpr int kBallots = (NW * kSlots + 31) / 32;
           unsigned bal[kBallots];
           int live = 0;
-#pragma unroll
-          for (int b = 0; b < kBallots; ++b) {
-            bal[b] = vote(b);
-            unsigned t = bal[b];                             // folded to one bit per live worker
-            t |= t >> 1;
-            t |= t >> 2;
-            if (kSlots >= 8) t |= t >> 4;
-            if (kSlots >= 16) t |= t >> 8;
-            live += __popc(t & (kSlots == 4 ? 0x11111111u : kSlots == 8 ? 0x01010101u : 0x00010001u));
-          }
           bool done = false;
-          if constexpr (GB == 2 && NW <= 32) {
+          if (all_live_left > 0) {
+            // Every worker was live in the last tile looked at (dense codes, as always with the
+            // moments on the workers): decoding a worker that has nothing to add is harmless
+            // (+0), so for 8, 16, ... 256 tiles the vote itself is left out.
+            --all_live_left;
+#pragma unroll kUnroll
+            for (int i = 0; i < NW; ++i) contribute(i);
+            done = true;
+          } else {
+#pragma unroll
+            for (int b = 0; b < kBallots; ++b) {
+              bal[b] = vote(b);
+              unsigned t = bal[b];                             // folded to one bit per live worker
+              t |= t >> 1;
+              t |= t >> 2;
+              if (kSlots >= 8) t |= t >> 4;
+              if (kSlots >= 16) t |= t >> 8;
+              live += __popc(t & (kSlots == 4 ? 0x11111111u : kSlots == 8 ? 0x01010101u : 0x00010001u));
+            }
+            if (live == NW) {
+              all_live_span = all_live_span < 256 ? 2 * all_live_span : 256;
+              all_live_left = all_live_span;
+            } else {
+              all_live_span = 4;
+            }
+          }
+          if constexpr (GB == 2 && NW <= 32) if (!done) {
             // Between "a few live workers" and "codes everywhere": a live worker still has
             // level 0 in nearly all of its bytes.  Each lane notes, per row, which live workers
             // have anything in ITS byte; the warp then works in rounds, lane by lane taking its
