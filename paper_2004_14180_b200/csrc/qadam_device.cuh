@@ -211,6 +211,64 @@ __device__ __forceinline__ unsigned quantize_grad(float u, const GradScale& gs, 
   return (unsigned)(neg ? L - c : L + c);
 }
 
+// A lane's 4 two-bit codes, given as one byte, stored as part of its warp's row of 128 codes
+// (32 bytes): two shuffle steps gather four lanes' bytes into a word, which lanes 0, 4, ..., 28
+// store.  Every lane of the warp must call this.  row_dst: address of the row's first code.
+__device__ __forceinline__ void store_row_of_code_bytes(unsigned byte, void* row_dst, int lane) {
+  unsigned w = byte | (__shfl_down_sync(0xffffffffu, byte, 1) << 8);
+  w |= __shfl_down_sync(0xffffffffu, w, 2) << 16;
+  if ((lane & 3) == 0) reinterpret_cast<unsigned*>(row_dst)[lane >> 2] = w;
+}
+
+// sat(d * 2^127): 1 for every positive d >= 2^-127 (every positive float difference the callers
+// form), 0 for zero, negative values and NaN.  One instruction on the fp32 pipe in place of a
+// comparison and a select on the integer pipe.
+__device__ __forceinline__ float positive_as_one(float d) {
+  float r;
+  asm("mul.rn.sat.f32 %0, %1, 0f7F000000;" : "=f"(r) : "f"(d));
+  return r;
+}
+
+// Ternary Q_g of 4 consecutive coordinates of one lane, the error update, and the lane's byte of
+// packed codes (code = level index + 1, coordinate c in bits 2c, 2c + 1).  Same decisions as
+// quantize_grad<G_TERNARY>: level 1 iff fl(|u| / s) > 1/2, settled without dividing outside the
+// sliver (s/2, (s/2)(1 + 2^-21)], by the division inside it and for scales that are not ordinary
+// numbers.  Outside the sliver everything runs on the fp32 pipe (the integer pipe, at half its
+// rate, is what the quantize kernels are otherwise bound by): [|u| > t] is sat((|u| - t) 2^127),
+// exact because the difference of two nearby floats is exact and at least 2^-125 for the scales
+// that take this path; the codes are gathered by exact multiply-adds and read out of a mantissa.
+__device__ __forceinline__ unsigned quantize_ternary4(const float (&u)[4], const GradScale& gs, float (&e_next)[4]) {
+  const float s = gs.s;
+  float up[4];
+  if (gs.fast) {
+    float band = 0.0f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const float a = fabsf(u[c]);
+      up[c] = positive_as_one(__fsub_rn(a, gs.half_hi));
+      band = __fadd_rn(band, __fsub_rn(positive_as_one(__fsub_rn(a, gs.half)), up[c]));
+    }
+    if (band != 0.0f) {                       // some |u| lies inside the sliver: the division decides
+#pragma unroll
+      for (int c = 0; c < 4; ++c) up[c] = __fdiv_rn(fabsf(u[c]), s) > 0.5f ? 1.0f : 0.0f;
+    }
+  } else {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) up[c] = __fdiv_rn(fabsf(u[c]), s) > 0.5f ? 1.0f : 0.0f;
+  }
+  float cf[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const float sign1 = __uint_as_float((__float_as_uint(u[c]) & 0x80000000u) | 0x3f800000u);   // +-1 with u's sign
+    // up * (+-s) + (+0): +-s for level +-1 and +0 (never -0) for level 0, as the definition has it
+    const float deq = __fmaf_rn(up[c], __fmul_rn(sign1, s), 0.0f);
+    e_next[c] = __fsub_rn(u[c], deq);
+    cf[c] = __fmaf_rn(up[c], sign1, 1.0f);                                                     // 0, 1 or 2
+  }
+  const float packed = __fmaf_rn(__fmaf_rn(__fmaf_rn(cf[3], 4.0f, cf[2]), 4.0f, cf[1]), 4.0f, cf[0]);
+  return __float_as_uint(__fadd_rn(packed, 8388608.0f)) & 0xffu;
+}
+
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3",
 // SC 2011), from its published definition: ten rounds over a counter of four 32-bit words
 // under a key of two; a round multiplies words 0 and 2 by fixed odd constants, keeps both

@@ -290,7 +290,7 @@ worker_absmax_kernel(const WorkerParams p) {
 // packed; e <- u - Q_g(u).  U_IN_E: u was left in e's slot by phase 1.
 // ---------------------------------------------------------------------------
 template <bool U_IN_E, int MODE, bool L2 = false>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, L2 ? 3 : 1)
 worker_quantize_kernel(const WorkerParams p) {
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
   // Tiles per round of loads, then of arithmetic and stores.  (Two per round when only e is
@@ -359,6 +359,8 @@ worker_quantize_kernel(const WorkerParams p) {
           code[1] = quantize_grad_stochastic(uu[1], s, rnd.y, en[1]);
           code[2] = quantize_grad_stochastic(uu[2], s, rnd.z, en[2]);
           code[3] = quantize_grad_stochastic(uu[3], s, rnd.w, en[3]);
+        } else if constexpr (MODE == G_TERNARY) {
+          code[0] = quantize_ternary4(uu, gs, en);           // the lane's byte of four codes
         } else {
 #pragma unroll
           for (int c = 0; c < 4; ++c) code[c] = quantize_grad<MODE>(uu[c], gs, p.k, p.L, en[c]);
@@ -366,7 +368,9 @@ worker_quantize_kernel(const WorkerParams p) {
         st_f4(p.e + so + idx, make_float4(en[0], en[1], en[2], en[3]));
         const long long row_elem = tile[a].off + r * kRowElems + warp * 128;
         void* dst = cw + row_elem * p.bits / 8;
-        if constexpr (MODE == G_TERNARY || MODE == G_STOCHASTIC) {
+        if constexpr (MODE == G_TERNARY) {
+          store_row_of_code_bytes(code[0], dst, lane);
+        } else if constexpr (MODE == G_STOCHASTIC) {
           pack_row_store<2>(code[0], code[1], code[2], code[3], dst, lane);
         } else if constexpr (MODE == G_FIVE) {
           pack_row_store<3>(code[0], code[1], code[2], code[3], dst, lane);

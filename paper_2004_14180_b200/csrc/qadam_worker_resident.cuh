@@ -529,13 +529,17 @@ worker_resident_kernel(const WorkerResidentParams rp) {
         const float uu[4] = {u4[r].x, u4[r].y, u4[r].z, u4[r].w};
         unsigned code[4];
         float en[4];
+        if constexpr (MODE == G_TERNARY) {
+          code[0] = quantize_ternary4(uu, gs, en);             // the lane's byte of four codes
+        } else {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) code[c] = quantize_grad<MODE>(uu[c], gs, p.k, p.L, en[c]);
+          for (int c = 0; c < 4; ++c) code[c] = quantize_grad<MODE>(uu[c], gs, p.k, p.L, en[c]);
+        }
         *reinterpret_cast<float4*>(ew + q * kRowElems) = make_float4(en[0], en[1], en[2], en[3]);
         const long long row_elem = cd.off + q * kRowElems + gwarp * 128;
         void* dst = cw + row_elem * p.bits / 8;
         if constexpr (MODE == G_TERNARY) {
-          pack_row_store<2>(code[0], code[1], code[2], code[3], dst, lane);
+          store_row_of_code_bytes(code[0], dst, lane);
         } else if constexpr (MODE == G_FIVE) {
           pack_row_store<3>(code[0], code[1], code[2], code[3], dst, lane);
         } else {
