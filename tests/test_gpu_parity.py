@@ -579,3 +579,38 @@ def test_weight_feedback_buffer(kx, n, kg, placement):
     with pytest.raises(qb.QAdamError) as ei:
         qb.QAdam([1000], 2, kg=0, kx=-1, want_wfeedback=True)      # nothing to feed back without Q_x
     assert ei.value.code == -3
+
+
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_ternary_decision_around_the_sliver_and_at_the_ends_of_the_fast_range(placement):
+    """The ternary level is decided without a division outside the sliver (s/2, (s/2)(1 + 2^-21)]
+    and by saturating fp32 differences: every float within 12 ulps of both ends of the sliver,
+    both signs, for an ordinary scale, for scales at the two ends of the range that takes the
+    fast path (1.1e-30, 2.9e38) and just outside it (0.9e-30: the division decides everything)."""
+    d, n = 4096 + 512, 4
+    scales = np.array([1.0, 1.1e-30, 2.9e38, 0.9e-30], np.float32)
+    g = np.zeros((n, d), np.float32)
+    rng = np.random.default_rng(5 + placement)
+    for i, s in enumerate(scales):
+        half = np.float32(0.5) * s
+        hi = half * np.float32(1.0 + 2.0 ** -21)
+        vals = []
+        for base in (half, hi):
+            v = base
+            for _ in range(12):
+                v = np.nextafter(v, np.float32(0))
+            for _ in range(25):
+                vals.append(v)
+                v = np.nextafter(v, np.float32(np.inf))
+        vals = np.array(vals, np.float32)
+        row = rng.choice(np.concatenate([vals, -vals, np.float32([0.0]), half * np.float32([0.25, 0.9, 1.5, 1.99])]), d)
+        row[0] = s                                           # the scale itself
+        g[i] = row.astype(np.float32)
+    p = Pair([d], n, 0, 0, placement, x1=np.zeros(d, np.float32))
+    if placement == S_MODE:
+        p.step(g)                                            # u = g exactly (e = 0)
+        p.compare_state()
+        assert np.array_equal(p.cpu.scales[:, 0], scales)
+    p.step(g)
+    p.compare_state()
+    p.close()
