@@ -341,17 +341,6 @@ WorkerResidentKernel pick_worker_resident(const qadam_ctx* c, bool l2, bool word
   }
 }
 
-// With the l2 term, the moments on the server and held weights that are not packed codes
-// of at most 8 bits, the streaming launches run instead of the on-chip kernel: its 8
-// load-side warps would fetch the held weights from global memory with nothing to hide the
-// latency behind, and lose (measured).  Packed codes of at most 8 bits are fetched a tile
-// ahead; with the moments on the workers the load side has 16 warps and more arithmetic
-// per element, and the on-chip kernel wins either way.
-bool l2_split(const qadam_ctx* c) {
-  return c->lambda != 0.0f && c->cfg.placement == QADAM_PLACE_SERVER &&
-         !(c->cfg.kx >= 0 && c->geo.xbits <= 8);
-}
-
 // grids of the split worker kernels (they depend on whether the l2 term is on)
 bool plan_worker_grids(qadam_ctx* c) {
   const int a = resident_grid(pick_absmax(c), 0, c->sm_count);
@@ -703,7 +692,7 @@ int qadam_worker_compress(qadam_ctx* c, int64_t step, const float* g,
     if (!cuda_ok(cudaMemsetAsync(p.scale_bits + (size_t)worker_begin * p.S, 0,
                                  sizeof(unsigned) * (size_t)worker_count * p.S, c->stream)))
       return QADAM_ERR_CUDA;
-    bool on_chip = c->grid_resident > 0 && !l2_split(c);
+    bool on_chip = c->grid_resident > 0;
     if (on_chip) {
       const size_t pairs = (size_t)c->cfg.n * p.S;     // all pairs' records are cleared, the call's are used
       const bool l2 = c->lambda != 0.0f;
@@ -952,7 +941,7 @@ int qadam_profile_read(qadam_ctx* c, double* ms, int64_t* launches) {
 
 int qadam_worker_pass_model(const qadam_ctx* c, int64_t* one_pass, int64_t* two_pass) {
   if (!c || !one_pass || !two_pass) return QADAM_ERR_NULL;
-  if (c->grid_resident > 0 && !l2_split(c)) {
+  if (c->grid_resident > 0) {
     *one_pass = (int64_t)c->cfg.n * c->geo.resident_elems;
     *two_pass = (int64_t)c->cfg.n * (c->geo.D - c->geo.resident_elems);
   } else {

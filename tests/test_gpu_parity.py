@@ -268,8 +268,7 @@ def test_on_chip_worker_capacity_boundary(placement):
 def test_on_chip_worker_l2_term_many_tiles(kx, placement):
     # the l2 term inside the on-chip kernel with several tiles per CTA: the held-weight
     # codes of a tile are fetched while the tile before it is processed (widths up to 8
-    # bits); wider codes and unquantized weights are read in place or take the streaming
-    # launches
+    # bits); wider codes and unquantized weights are read in place
     sms = torch.cuda.get_device_properties(0).multi_processor_count
     seg = [sms * 3 * 4096 + 300, 5000, 70000, 129]
     n, d = 3, sum([sms * 3 * 4096 + 300, 5000, 70000, 129])
@@ -581,16 +580,17 @@ def test_weight_feedback_buffer(kx, n, kg, placement):
     assert ei.value.code == -3
 
 
-@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
-def test_ternary_decision_around_the_sliver_and_at_the_ends_of_the_fast_range(placement):
+def test_ternary_decision_around_the_sliver_and_at_the_ends_of_the_fast_range():
     """The ternary level is decided without a division outside the sliver (s/2, (s/2)(1 + 2^-21)]
     and by saturating fp32 differences: every float within 12 ulps of both ends of the sliver,
     both signs, for an ordinary scale, for scales at the two ends of the range that takes the
-    fast path (1.1e-30, 2.9e38) and just outside it (0.9e-30: the division decides everything)."""
+    fast path (1.1e-30, 2.9e38) and just outside it (0.9e-30: the division decides everything).
+    Worker side only, moments on the server, e = 0, so that u is exactly the value planted (the
+    server's average of such scales would overflow)."""
     d, n = 4096 + 512, 4
     scales = np.array([1.0, 1.1e-30, 2.9e38, 0.9e-30], np.float32)
     g = np.zeros((n, d), np.float32)
-    rng = np.random.default_rng(5 + placement)
+    rng = np.random.default_rng(5)
     for i, s in enumerate(scales):
         half = np.float32(0.5) * s
         hi = half * np.float32(1.0 + 2.0 ** -21)
@@ -606,11 +606,17 @@ def test_ternary_decision_around_the_sliver_and_at_the_ends_of_the_fast_range(pl
         row = rng.choice(np.concatenate([vals, -vals, np.float32([0.0]), half * np.float32([0.25, 0.9, 1.5, 1.99])]), d)
         row[0] = s                                           # the scale itself
         g[i] = row.astype(np.float32)
-    p = Pair([d], n, 0, 0, placement, x1=np.zeros(d, np.float32))
-    if placement == S_MODE:
-        p.step(g)                                            # u = g exactly (e = 0)
-        p.compare_state()
+    for options in (None, "streaming"):
+        import paper_2004_14180_b200 as qb
+        opt = qb.QAdamOptions(worker_kernel=qb.WORKER_STREAMING) if options else None
+        p = Pair([d], n, 0, 0, S_MODE, x1=np.zeros(d, np.float32), options=opt)
+        gp = p.cpu.to_padded(g)
+        p.gpu.worker_compress(1, torch.from_numpy(gp).cuda())
+        p.cpu.workers_step(gp, p.lr)
+        p.compare_worker_outputs()
         assert np.array_equal(p.cpu.scales[:, 0], scales)
-    p.step(g)
-    p.compare_state()
-    p.close()
+        assert bits_equal(p.gpu.e.cpu().numpy(), p.cpu.e), "e differs"
+        # some values of every worker fall on either side, and inside the sliver
+        codes = p.cpu.gcodes
+        assert (codes != 0x55).any(axis=1).all()
+        p.close()
