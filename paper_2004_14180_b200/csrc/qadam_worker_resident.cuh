@@ -30,7 +30,9 @@
 // pair records in global memory and the slots' "free" barriers: the load side runs
 // ahead of the store side by as many tiles as there are slots, which is what hides the
 // latency of the grid-wide hand-over (last load of a pair lands somewhere -> every CTA
-// learns the scale).  No deadlock: a load waits for the store of the tile `slots`
+// learns the scale).  A pair of a single tile (a bias vector, a block of a block-wise
+// scale that fits one tile) skips the global record: the dispatcher takes the maximum
+// from the tile's header in shared memory.  No deadlock: a load waits for the store of the tile `slots`
 // places earlier in the same CTA, which waits for that tile's pair to be complete, which
 // waits for loads of that pair only; a pair gives a CTA fewer tiles than it has slots
 // (the host sends larger pairs elsewhere), so those loads wait, in turn, only for
@@ -103,7 +105,8 @@ struct RLoadHeader {       // one per tile in flight on the load side (ring of k
   long long pair;          // worker * S + segment
   int slot;                // where g lands and u stays
   int count;               // elements of the tile
-  int publish;             // last tile of the CTA's streak of this pair
+  int publish;             // 1: last tile of the CTA's streak of this pair; 2: the pair is this one tile and
+                           // is handed over inside the CTA (nothing to publish or to count)
   unsigned max_bits;       // max |u| of the tile, folded in by the consumer warps
   long long elem;          // worker * D + first element: where m, v go back (moments on the workers)
   long long off;           // first element in the vector: where the held weights are (l2 term)
@@ -198,7 +201,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
       RTile next = cur;
       const bool has_next = i + 1 < my_tiles;
       if (has_next) next = rp.rtiles[jn];
-      const int publish = !(has_next && worker_n == worker && next.seg == cur.seg);
+      const int publish = cur.need == 1 ? 2 : !(has_next && worker_n == worker && next.seg == cur.seg);
       if (lane == 0) {
         // the slot must have been read out by the store side (a fresh barrier passes a wait on
         // the parity opposite to its first phase), the ring stage by the consumers
@@ -262,6 +265,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
         const int hi = (int)(i & (kRHeaders - 1));
         if (!mbar_wait_bounded(&ps->hd_ready[hi], (unsigned)(i / kRHeaders) & 1u, abort_flag, p.status, spin)) break;
         const RLoadHeader hd = ps->load_hd[hi];
+        if (hd.publish == 2) continue;                   // a one-tile pair: the dispatcher reads the header itself
         acc_max = max(acc_max, hd.max_bits);
         acc_cnt += 1;
         if (WORDS && hd.publish) {
@@ -299,7 +303,24 @@ worker_resident_kernel(const WorkerResidentParams rp) {
         const long long pair = (long long)(p.worker_begin + worker) * p.S + cur.seg;
         if (pair != ready_pair) {                        // warp-uniform
           ok = false;
-          if constexpr (WORDS) {
+          if (cur.need == 1) {
+            // The pair is this one tile, which this CTA loaded: its maximum is complete in the
+            // tile's header once the load-side warps have arrived there, and nothing has to
+            // cross to another CTA.  The header is still the tile's own: the load side runs at
+            // most `slots` tiles ahead of this warp, fewer than the ring of headers holds, and
+            // for the same reason the barrier's phase is the one the tile armed.
+            const int hi = (int)(i & (kRHeaders - 1));
+            if (lane == 0) {
+              ok = mbar_wait_bounded(&ps->hd_ready[hi], (unsigned)(i / kRHeaders) & 1u, abort_flag, p.status, spin);
+              if (ok) {
+                ready_scale = ps->load_hd[hi].max_bits;
+                p.scale_bits[pair] = ready_scale;
+                if (ready_scale >= 0x7f800000u) atomicOr(p.status, 1u);
+              }
+            }
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            ready_scale = __shfl_sync(0xffffffffu, ready_scale, 0);
+          } else if constexpr (WORDS) {
             // the whole warp gathers the words of the CTAs that hold tiles of the pair:
             // CTAs (t0 + k) mod ctas, k < min(need, ctas), t0 the pair's first tile
             const long long t0 = (long long)worker * rp.TR + cur.first;

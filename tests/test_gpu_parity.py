@@ -294,6 +294,32 @@ def test_on_chip_worker_counter_hand_over(placement):
          options=qb.QAdamOptions(hand_over=qb.HANDOVER_COUNTERS))
 
 
+@pytest.mark.parametrize("hand_over", ["auto", "counters"])
+@pytest.mark.parametrize("placement", [S_MODE, W_MODE])
+def test_on_chip_worker_one_tile_pairs(placement, hand_over):
+    # pairs of a single tile take their scale from the tile's header inside the CTA; here
+    # each CTA gets more than 32 of them in a row (the ring of headers goes round), with
+    # pairs of several tiles in between, with and without the l2 term
+    import paper_2004_14180_b200 as qb
+    sms = torch.cuda.get_device_properties(0).multi_processor_count
+    sizes = (4096, 2048, 100, 4095, 1)
+    seg = [sizes[k % len(sizes)] for k in range(sms * 34)]
+    seg[sms * 7] = 3 * 4096 + 5
+    seg[sms * 20 + 3] = sms * 4096 + 77
+    n, d = 2, sum(seg)
+    rng = np.random.default_rng(120 + placement)
+    x1 = (rng.standard_normal(d) * 0.3).astype(np.float32)
+    opt = qb.QAdamOptions(hand_over=qb.HANDOVER_COUNTERS) if hand_over == "counters" else None
+    p = Pair(seg, n, 0, 0, placement, x1=x1, options=opt)
+    one, two = p.gpu.worker_pass_model()
+    assert two == 0, "every pair fits on chip"
+    for lam in (0.0, 5e-4):
+        p.set_regularization(lam)
+        p.step(_rand_grads(rng, n, d))
+        p.compare_state()
+    p.close()
+
+
 @pytest.mark.parametrize("placement", [S_MODE, W_MODE])
 def test_streaming_launches_only(placement):
     # worker_kernel = STREAMING sends every pair through the two streaming launches, the
