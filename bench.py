@@ -81,6 +81,8 @@ def parse_args():
                     help="one max-abs scale per block of 2^K elements of a tensor (0: per tensor)")
     ap.add_argument("--weight-decay", type=float, default=0.0,
                     help="lambda of the l2 term g + lambda * (held weights); 0: none")
+    ap.add_argument("--weight-feedback", action="store_true",
+                    help="give the weight broadcast an error buffer of its own (Q_x applied to x + e^w)")
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -170,7 +172,7 @@ class ClockSampler:
 # ----------------------------------------------------------------------------- byte accounting
 
 def algorithmic_bytes(kernel: str, w, placement: str, D: int, gbits: int, xbits: int,
-                      pass_model=None, l2_term: bool = False) -> float:
+                      pass_model=None, l2_term: bool = False, weight_feedback: bool = False) -> float:
     """Bytes one launch of `kernel` must move at its interface (fp32 state it has
     to read and write, packed codes), for all n workers.  The worker side is capacity
     aware: (worker, segment) pairs that fit on chip go through the fused kernel and are
@@ -197,6 +199,8 @@ def algorithmic_bytes(kernel: str, w, placement: str, D: int, gbits: int, xbits:
         return per * n * D
     if kernel == "server":      # read n code streams and x (m, v); write x (m, v) and the broadcast
         state = 24.0 if server_moments else 8.0
+        if weight_feedback:     # the broadcast's own error buffer is read and written too
+            state += 8.0
         return (n * gbits / 8.0 + state + xbits / 8.0) * D
     if kernel == "broadcast":
         return (4.0 + xbits / 8.0) * D
@@ -258,6 +262,7 @@ def workload_config(w, args, extra=None):
         "workload": f"{w.name} (d={w.d}, {w.num_segments} scale segment(s), n={w.n} workers)",
         "d": w.d, "n_workers": w.n, "segments": w.num_segments,
         "kg": w.kg, "kx": w.kx, "placement": args.placement, "weight_decay": args.weight_decay,
+        "weight_feedback": bool(getattr(args, "weight_feedback", False)),
         "beta1": w.beta1, "beta2": w.beta2, "eps": w.eps, "lr": w.lr,
         "gradients": w.grad, "parallelism": f"replicas x{args.gpus} (no exchange between GPUs)",
         "l2": ("inputs larger than L2 (no flush between steps)" if 8 * w.n * w.d > (1 << 28) else
@@ -311,7 +316,7 @@ def alu_decode_peak():
     return props.multi_processor_count * 64.0 * mhz * 1e6
 
 
-def kernel_table(prof, w, placement_name, q, weight_decay, peak):
+def kernel_table(prof, w, placement_name, q, weight_decay, peak, weight_feedback=False):
     """Per kernel: launches, time, algorithmic bytes, achieved rate and its fractions."""
     D = q.D
     kernels = {}
@@ -321,7 +326,8 @@ def kernel_table(prof, w, placement_name, q, weight_decay, peak):
             continue
         per = ms / cnt
         bytes_ = algorithmic_bytes(name, w, placement_name, D, q.gcode_bytes * 8 // D, q.wcode_bytes * 8 // D,
-                                   pass_model=q.worker_pass_model(), l2_term=weight_decay != 0.0)
+                                   pass_model=q.worker_pass_model(), l2_term=weight_decay != 0.0,
+                                   weight_feedback=weight_feedback)
         gbs = bytes_ / (per * 1e-3) / 1e9
         kernels[name] = {"launches": int(cnt), "ms_per_launch": per, "share": ms / total_ms,
                          "algorithmic_bytes": bytes_, "achieved_gbs": gbs,
@@ -338,7 +344,8 @@ def kernel_table(prof, w, placement_name, q, weight_decay, peak):
 class Measured:
     """One workload set up on the device and timed: the context stays open for the caller."""
 
-    def __init__(self, w, placement_name, weight_decay, steps, warmup, dev, world, peak, sample_clocks):
+    def __init__(self, w, placement_name, weight_decay, steps, warmup, dev, world, peak, sample_clocks,
+                 weight_feedback=False):
         import torch
         import torch.distributed as dist
         import qadam_inputs as qi
@@ -347,7 +354,7 @@ class Measured:
         placement = qb.PLACE_SERVER if placement_name == "server" else qb.PLACE_WORKER
         x1 = qi.initial_weights(w, dev)
         q = qb.QAdam(w.scale_seg_len, w.n, kg=w.kg, kx=w.kx, placement=placement, beta1=w.beta1,
-                     beta2=w.beta2, eps=w.eps, lr=w.lr, x1=x1, device=dev)
+                     beta2=w.beta2, eps=w.eps, lr=w.lr, x1=x1, device=dev, want_wfeedback=weight_feedback)
         q.set_regularization(weight_decay)
         del x1
         self.q, D = q, q.D
@@ -394,7 +401,7 @@ class Measured:
         self.status = q.poll_status()
         self.ms_step = max_over_ranks(ms_total, world, dev) / steps
         self.value = job_value(w.d, w.n, world, self.ms_step)
-        self.kernels = kernel_table(prof, w, placement_name, q, weight_decay, peak)
+        self.kernels = kernel_table(prof, w, placement_name, q, weight_decay, peak, weight_feedback)
         self.step_bytes = sum(k["algorithmic_bytes"] * k["launches"] for k in self.kernels.values()) / steps
 
     def close(self):
@@ -404,10 +411,12 @@ class Measured:
 
 
 # The configurations reported beside the headline: both large workloads over the worker-count
-# sweep, the ResNet-18-shaped sets, both placements of the moments, one run with the l2 term.
+# sweep, the ResNet-18-shaped sets, both placements of the moments, one run with the l2 term,
+# and (a fifth field) two with an error buffer of its own for the weight broadcast.
 CONFIG_RUNS = (
     ("bert_base", None, "server", 0.0), ("bert_base", None, "worker", 0.0),
     ("bert_base", None, "server", 5e-4),
+    ("bert_base", None, "server", 0.0, True), ("flat28", 16, "server", 0.0, True),
     ("flat28", 1, "server", 0.0), ("flat28", 4, "server", 0.0), ("flat28", 32, "server", 0.0),
     ("flat28", 1, "worker", 0.0), ("flat28", 4, "worker", 0.0), ("flat28", 16, "worker", 0.0),
     ("flat28", 32, "worker", 0.0),
@@ -423,17 +432,19 @@ def config_records(args, dev, world, peak):
     import qadam_inputs as qi
     out = []
     free_b, _total = torch.cuda.mem_get_info(dev)
-    for name, n, placement_name, wd in CONFIG_RUNS:
+    for name, n, placement_name, wd, *more in CONFIG_RUNS:
+        wf = bool(more and more[0])
         w = qi.get_workload(name, n=n)
         # g, e (and the workers' m, v) dominate; skip what this device cannot hold
         need = w.n * w.d * 4 * (4 if placement_name == "worker" else 2) + 4 * w.d * 4
         rec = {"workload": w.name, "n_workers": w.n, "placement": placement_name, "weight_decay": wd,
-               "kg": w.kg, "kx": w.kx, "d": w.d, "segments": w.num_segments}
+               "weight_feedback": wf, "kg": w.kg, "kx": w.kx, "d": w.d, "segments": w.num_segments}
         if need > 0.92 * free_b:
             rec["skipped"] = f"needs {need >> 30} GiB of {free_b >> 30} GiB free"
             out.append(rec)
             continue
-        m = Measured(w, placement_name, wd, args.config_steps, 3, dev, world, peak, sample_clocks=True)
+        m = Measured(w, placement_name, wd, args.config_steps, 3, dev, world, peak, sample_clocks=True,
+                     weight_feedback=wf)
         rec.update({"ms_per_step": m.ms_step, "value": m.value, "unit": UNIT, "steps": args.config_steps,
                     "device_status": int(m.status), "clocks": m.clock_info,
                     "step_frac": m.step_bytes / (m.ms_step * 1e-3) / 1e9 / peak,
@@ -468,7 +479,7 @@ def run_b200(args):
     w = get_workload(args)
     peak, peak_kind = measured_peak()
     m = Measured(w, args.placement, args.weight_decay, args.steps, args.warmup, dev, world, peak,
-                 sample_clocks=True)
+                 sample_clocks=True, weight_feedback=args.weight_feedback)
     q, g, D = m.q, m.g, m.q.D
     if w.n * D * 4 <= (1 << 27):
         print(f"note: gradient input is {w.n * D * 4 >> 20} MiB, not larger than L2", file=sys.stderr)

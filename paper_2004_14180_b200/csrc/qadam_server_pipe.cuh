@@ -333,13 +333,15 @@ __host__ __device__ constexpr int vote_pieces_pow2(int gb) { return gb <= 2 ? 2 
 // packed store of the warp's row of 128 two-bit codes (32 bytes): the four codes of a lane
 // are one byte; two shuffle steps gather four lanes' bytes into a word, which lanes
 // 0, 4, ..., 28 store.  row_dst: address of the row's first code.
-// wfeedback_elem (optional): the thread's 4 values of the broadcast's error buffer, see broadcast_row.
+// wfeedback_elem (optional): the thread's 4 values of the broadcast's error buffer, see broadcast_row;
+// ew_fetched (optional): their old contents, read by the caller ahead of time.
 __device__ __forceinline__ void broadcast_row_ternary(const float xin[4], unsigned char* row_dst,
-                                                      float* wresid_elem, float* wfeedback_elem, int lane) {
+                                                      float* wresid_elem, float* wfeedback_elem,
+                                                      const float4* ew_fetched, int lane) {
   float xx[4] = {xin[0], xin[1], xin[2], xin[3]};
   float xq[4];
   if (wfeedback_elem) {
-    const float4 ew = ld_f4(wfeedback_elem);
+    const float4 ew = ew_fetched ? *ew_fetched : ld_f4(wfeedback_elem);
     xx[0] = __fadd_rn(xx[0], ew.x); xx[1] = __fadd_rn(xx[1], ew.y);
     xx[2] = __fadd_rn(xx[2], ew.z); xx[3] = __fadd_rn(xx[3], ew.w);
   }
@@ -578,6 +580,16 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
       auto active = [&](int r) { return r * kPipeRowElems + gt * 4 < hd.count; };   // monotone in r
       float2 a[2 * ROWS];
       float4 x4[ROWS], m4[ROWS], v4[ROWS];
+      // the broadcast's own error buffer (optional) is not staged: its values are asked for
+      // now and used after the decode, which hides the latency of the plain loads (where the
+      // registers allow: two-row tiles with the ternary broadcast; elsewhere they are read in place)
+      constexpr bool kFetchEwAhead = XB == 2 && ROWS == 2;
+      float4 ew4[ROWS];
+      if (kFetchEwAhead && p.wfeedback != nullptr && act0) {
+#pragma unroll
+        for (int r = 0; r < ROWS; ++r)
+          if (active(r)) ew4[r] = ld_f4(p.wfeedback + hd.off + r * kPipeRowElems + gt * 4);
+      }
       if (act0) {
         // ternary: the thread's byte of a row; five levels: the first of its two bytes
         // (table decode: the first byte of the warp's packed row)
@@ -795,7 +807,8 @@ server_pipe_kernel(const ServerParams p, const __grid_constant__ CUtensorMap cod
           if constexpr (XB == 2) {
             broadcast_row_ternary(xx, p.wcodes + ((e0 + gwarp * 128) >> 2),
                                   p.wresid ? p.wresid + e0 + gt * 4 : nullptr,
-                                  p.wfeedback ? p.wfeedback + e0 + gt * 4 : nullptr, lane);
+                                  p.wfeedback ? p.wfeedback + e0 + gt * 4 : nullptr,
+                                  kFetchEwAhead ? &ew4[r] : nullptr, lane);
           } else {
             if (p.kx >= 0)
               broadcast_row(xx, p.kx, p.xbits, p.wcodes, p.wresid, p.wfeedback, e0 + gt * 4, e0 + gwarp * 128, lane);
