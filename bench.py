@@ -422,6 +422,8 @@ CONFIG_RUNS = (
     ("flat28", 32, "worker", 0.0),
     ("resnet18_qg", None, "server", 0.0), ("resnet18_qg", None, "worker", 0.0),
     ("resnet18_qg_qx_k0", None, "server", 0.0), ("resnet18_qg_qx_k0", None, "worker", 0.0),
+    ("resnet18_qg_qx_k1", None, "server", 0.0), ("resnet18_qg_qx_k1", None, "worker", 0.0),
+    ("flat20", None, "server", 0.0), ("flat20", None, "worker", 0.0),
 )
 
 
