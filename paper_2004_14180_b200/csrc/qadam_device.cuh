@@ -269,6 +269,55 @@ __device__ __forceinline__ unsigned quantize_ternary4(const float (&u)[4], const
   return __float_as_uint(__fadd_rn(packed, 8388608.0f)) & 0xffu;
 }
 
+// Five-level Q_g (levels 0, 1/2, 1 times the scale, k_g = 1 of the geometric grid) of 4
+// consecutive coordinates of one lane, the error update, and the lane's 12 bits of packed codes
+// (code = level index + 2, coordinate c in bits 3c .. 3c + 2).  Same decisions as
+// quantize_grad<G_FIVE>: index [y > 1/4] + [y > 3/4] with y = fl(|u| / s).  y' = fl(|u| fl(1/s)) is
+// within 2^-22 (relative) of y, so y' above t (1 + 2^-20) or at most t (1 - 2^-20) settles the
+// comparison with the midpoint t; a y' in between sends the lane's four coordinates to the
+// division.  As in quantize_ternary4 the comparisons are saturated differences on the fp32 pipe
+// (a positive difference of y' and a threshold is at least 2^-26), the dequantized value is
+// index * (+-s/2), exact, and the codes are gathered by exact multiply-adds.
+__device__ __forceinline__ unsigned quantize_five4(const float (&u)[4], const GradScale& gs, float (&e_next)[4]) {
+  const float s = gs.s;
+  float idx[4];                                // level index 0, 1 or 2 as a float
+  bool divide = !gs.fast;
+  if (gs.fast) {
+    float band = 0.0f;
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const float yp = __fmul_rn(fabsf(u[c]), gs.inv);
+      const float up1 = positive_as_one(__fsub_rn(yp, 0.25000023841857910156f));     // 1/4 (1 + 2^-20)
+      const float lo1 = positive_as_one(__fsub_rn(yp, 0.24999976158142089844f));     // 1/4 (1 - 2^-20)
+      const float up3 = positive_as_one(__fsub_rn(yp, 0.75000071525573730469f));     // 3/4 (1 + 2^-20)
+      const float lo3 = positive_as_one(__fsub_rn(yp, 0.74999928474426269531f));     // 3/4 (1 - 2^-20)
+      idx[c] = __fadd_rn(up1, up3);
+      band = __fadd_rn(band, __fadd_rn(__fsub_rn(lo1, up1), __fsub_rn(lo3, up3)));
+    }
+    divide = band != 0.0f;
+  }
+  if (divide) {
+#pragma unroll
+    for (int c = 0; c < 4; ++c) {
+      const float y = __fdiv_rn(fabsf(u[c]), s);
+      idx[c] = (y > 0.25f ? 1.0f : 0.0f) + (y > 0.75f ? 1.0f : 0.0f);
+    }
+  }
+  float cf[4];
+#pragma unroll
+  for (int c = 0; c < 4; ++c) {
+    const float sign1 = __uint_as_float((__float_as_uint(u[c]) & 0x80000000u) | 0x3f800000u);   // +-1 with u's sign
+    // index * (+-s/2) + (+0): the level's value (s/2 and s are exact) and +0, never -0, for level 0.
+    // A scale so small that s/2 is not exact takes fl(s * level) as the definition has it.
+    const float deq = gs.fast ? __fmaf_rn(idx[c], __fmul_rn(sign1, gs.half), 0.0f)
+                              : (idx[c] == 0.0f ? 0.0f : __fmul_rn(__fmul_rn(s, __fmul_rn(0.5f, idx[c])), sign1));
+    e_next[c] = __fsub_rn(u[c], deq);
+    cf[c] = __fmaf_rn(idx[c], sign1, 2.0f);                                                     // 0 .. 4
+  }
+  const float packed = __fmaf_rn(__fmaf_rn(__fmaf_rn(cf[3], 8.0f, cf[2]), 8.0f, cf[1]), 8.0f, cf[0]);
+  return __float_as_uint(__fadd_rn(packed, 8388608.0f)) & 0xfffu;
+}
+
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw, "Parallel random numbers: as easy as 1, 2, 3",
 // SC 2011), from its published definition: ten rounds over a counter of four 32-bit words
 // under a key of two; a round multiplies words 0 and 2 by fixed odd constants, keeps both
@@ -334,6 +383,27 @@ __device__ __forceinline__ unsigned quantize_weight(float x, int kx, float& xq) 
 // ---------------------------------------------------------------------------
 __host__ __device__ constexpr int cgcd(int a, int b) { return b == 0 ? a : cgcd(b, a % b); }
 
+// The same for code widths up to 8 bits with the lane's four codes already gathered into one
+// field of 4 * B bits.
+template <int B>
+__device__ __forceinline__ void pack_row_store_fields(unsigned field, void* row_dst, int lane) {
+  static_assert(B >= 2 && B <= 8, "code width");
+  constexpr int F = 4 * B;                               // 8..32 bits per lane
+  constexpr int G = cgcd(32, F);
+  constexpr int J = (F - G + 32 + F - 1) / F;            // fields a 32-bit word can touch
+  const int bit0 = 32 * lane;
+  const int l0 = bit0 / F;
+  const int sh = bit0 - l0 * F;
+  unsigned long long acc = 0;
+#pragma unroll
+  for (int j = 0; j < J; ++j) {
+    const int src = l0 + j > 31 ? 31 : l0 + j;
+    const unsigned f = __shfl_sync(0xffffffffu, field, src);
+    acc |= (unsigned long long)f << (j * F);
+  }
+  if (lane < F) reinterpret_cast<unsigned*>(row_dst)[lane] = (unsigned)(acc >> sh);
+}
+
 template <int B>
 __device__ __forceinline__ void pack_row_store(unsigned c0, unsigned c1, unsigned c2, unsigned c3,
                                                void* row_dst, int lane) {
@@ -362,21 +432,7 @@ __device__ __forceinline__ void pack_row_store(unsigned c0, unsigned c1, unsigne
       if (w < F) reinterpret_cast<unsigned*>(row_dst)[w] = (unsigned)lo;
     }
   } else {
-    constexpr int F = 4 * B;                               // 8..32 bits per lane
-    constexpr int G = cgcd(32, F);
-    constexpr int J = (F - G + 32 + F - 1) / F;            // fields a 32-bit word can touch
-    const unsigned field = c0 | (c1 << B) | (c2 << (2 * B)) | (c3 << (3 * B));
-    const int bit0 = 32 * lane;
-    const int l0 = bit0 / F;
-    const int sh = bit0 - l0 * F;
-    unsigned long long acc = 0;
-#pragma unroll
-    for (int j = 0; j < J; ++j) {
-      const int src = l0 + j > 31 ? 31 : l0 + j;
-      const unsigned f = __shfl_sync(0xffffffffu, field, src);
-      acc |= (unsigned long long)f << (j * F);
-    }
-    if (lane < F) reinterpret_cast<unsigned*>(row_dst)[lane] = (unsigned)(acc >> sh);
+    pack_row_store_fields<B>(c0 | (c1 << B) | (c2 << (2 * B)) | (c3 << (3 * B)), row_dst, lane);
   }
 }
 

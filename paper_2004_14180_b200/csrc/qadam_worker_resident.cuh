@@ -554,6 +554,8 @@ worker_resident_kernel(const WorkerResidentParams rp) {
         float en[4];
         if constexpr (MODE == G_TERNARY) {
           code[0] = quantize_ternary4(uu, gs, en);             // the lane's byte of four codes
+        } else if constexpr (MODE == G_FIVE) {
+          code[0] = quantize_five4(uu, gs, en);                // the lane's 12 bits of four codes
         } else {
 #pragma unroll
           for (int c = 0; c < 4; ++c) code[c] = quantize_grad<MODE>(uu[c], gs, p.k, p.L, en[c]);
@@ -564,7 +566,7 @@ worker_resident_kernel(const WorkerResidentParams rp) {
         if constexpr (MODE == G_TERNARY) {
           store_row_of_code_bytes(code[0], dst, lane);
         } else if constexpr (MODE == G_FIVE) {
-          pack_row_store<3>(code[0], code[1], code[2], code[3], dst, lane);
+          pack_row_store_fields<3>(code[0], dst, lane);
         } else {
           pack_row_store_rt(p.bits, code[0], code[1], code[2], code[3], dst, lane);
         }

@@ -646,3 +646,43 @@ def test_ternary_decision_around_the_sliver_and_at_the_ends_of_the_fast_range():
         codes = p.cpu.gcodes
         assert (codes != 0x55).any(axis=1).all()
         p.close()
+
+
+def test_five_level_decision_around_both_midpoints_and_at_the_ends_of_the_fast_range():
+    """The five-level index [y > 1/4] + [y > 3/4] is settled from |u| * fl(1/s) by saturating
+    fp32 differences unless that product lies within 2^-20 (relative) of a midpoint, where the
+    division decides: every float within 12 ulps of s/4 and 3s/4 and of the two ends of either
+    band, both signs, for an ordinary scale, an awkward one (1/3: its reciprocal is rounded), and
+    scales at the two ends of the range that takes the fast path and just outside it.  Worker
+    side only, moments on the server, e = 0, so that u is exactly the value planted."""
+    import paper_2004_14180_b200 as qb
+    d, n = 4096 + 512, 5
+    scales = np.array([1.0, 1.0 / 3.0, 1.1e-30, 2.9e38, 0.9e-30], np.float32)
+    g = np.zeros((n, d), np.float32)
+    rng = np.random.default_rng(6)
+    for i, s in enumerate(scales):
+        vals = []
+        for t in (0.25, 0.75):
+            mid = np.float32(t) * s
+            for base in (mid * np.float32(1.0 - 2.0 ** -20), mid, mid * np.float32(1.0 + 2.0 ** -20)):
+                v = np.float32(base)
+                for _ in range(12):
+                    v = np.nextafter(v, np.float32(0))
+                for _ in range(25):
+                    vals.append(v)
+                    v = np.nextafter(v, np.float32(np.inf))
+        vals = np.array(vals, np.float32)
+        extra = s * np.float32([0.0, 0.1, 0.24, 0.26, 0.5, 0.74, 0.76, 0.99])
+        row = rng.choice(np.concatenate([vals, -vals, extra, -extra]), d)
+        row[0] = s                                           # the scale itself
+        g[i] = row.astype(np.float32)
+    for options in (None, "streaming"):
+        opt = qb.QAdamOptions(worker_kernel=qb.WORKER_STREAMING) if options else None
+        p = Pair([d], n, 1, 0, S_MODE, x1=np.zeros(d, np.float32), options=opt)
+        gp = p.cpu.to_padded(g)
+        p.gpu.worker_compress(1, torch.from_numpy(gp).cuda())
+        p.cpu.workers_step(gp, p.lr)
+        p.compare_worker_outputs()
+        assert np.array_equal(p.cpu.scales[:, 0], scales)
+        assert bits_equal(p.gpu.e.cpu().numpy(), p.cpu.e), "e differs"
+        p.close()
