@@ -328,6 +328,25 @@ worker_resident_kernel(const WorkerResidentParams rp) {
             const int kmax = cur.need < ctas ? cur.need : ctas;
             const unsigned long long* w = rp.words + pair * ctas;
             unsigned mx = 0;
+            if constexpr (WM) {
+              // With the moments on the workers the load side is the slower one, so a pair is
+              // rarely complete when the dispatcher first asks.  It then waits for the CTA that
+              // holds the pair's last tile, as a rule the last to publish, before it gathers: one
+              // word polled by one lane.  (All lanes polling all words of the pair is 1 KB per
+              // round and CTA, which takes a good part of the L2's bandwidth when many CTAs wait
+              // at once.)  Whatever this wait sees, the gather below decides.  With the moments on
+              // the server pairs are complete as a rule and the extra round trip costs more than
+              // it saves (measured both ways).
+              int c_last = c0 + (cur.need - 1) % ctas;
+              if (c_last >= ctas) c_last -= ctas;
+              if (lane == 0) {
+                for (unsigned it = 0; it < pair_spin; ++it) {
+                  if (ld_relaxed_u64(w + c_last) != 0ull || *abort_flag) break;
+                  __nanosleep(it < 64 ? 40 : 400);
+                }
+              }
+              __syncwarp();
+            }
             for (unsigned it = 0; it < pair_spin; ++it) {
               unsigned cnt = 0;
               mx = 0;
